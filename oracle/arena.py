@@ -1,0 +1,89 @@
+"""Offline static layout (Algorithm 1 of the paper) and the chunk-count search
+(test infrastructure only).
+
+Algorithm 1: visit tensors in descending size; for each, collect the already
+placed tensors whose lifetimes intersect its own, look at the address gaps those
+leave, take the smallest gap that holds the tensor, and otherwise place it above
+all of them.  Points the paper leaves open, fixed here:
+
+  * equal sizes are visited by (birth, death, id) ascending;
+  * lifetimes are half-open, [b_i, e_i) and [b_j, e_j) conflict iff
+    b_i < e_j and b_j < e_i;
+  * a gap is a finite hole between conflicting tensors in address order,
+    including the one that starts at address 0; equal-sized holes resolve to the
+    lowest address; the unbounded space above the highest conflict is not a gap
+    but the fallback position.
+
+Chunk search ("apply only as much mitigation as needed" with chunk count as the
+intensity): the smallest C in 1..max_chunks whose laid-out (reserved) peak is
+within the byte budget, found by a linear scan so no monotonicity is assumed.
+"""
+from __future__ import annotations
+
+from . import trace as _trace
+
+
+def conflicts(a, b):
+    return a["birth"] < b["death"] and b["birth"] < a["death"]
+
+
+def max_live_bytes(tensors, n_ops=None):
+    """max over op index t of the bytes of tensors with birth <= t < death."""
+    if not tensors:
+        return 0
+    n_ops = max(d["death"] for d in tensors) if n_ops is None else n_ops
+    best = 0
+    for t in range(n_ops):
+        live = sum(d["bytes"] for d in tensors if d["birth"] <= t < d["death"])
+        best = max(best, live)
+    return best
+
+
+def plan_arena(tensors):
+    """Returns (offsets, peak).  offsets[i] belongs to tensors[i]."""
+    n = len(tensors)
+    order = sorted(range(n), key=lambda i: (-tensors[i]["bytes"], tensors[i]["birth"], tensors[i]["death"], i))
+    offsets = [None] * n
+    placed = []
+    for i in order:
+        ti = tensors[i]
+        O = [j for j in placed if conflicts(ti, tensors[j])]
+        O.sort(key=lambda j: (offsets[j], j))
+        cursor = 0
+        best = None                      # (gap size, bottom address)
+        for j in O:
+            if offsets[j] > cursor:
+                gap = offsets[j] - cursor
+                if gap >= ti["bytes"] and (best is None or gap < best[0]):
+                    best = (gap, cursor)
+            cursor = max(cursor, offsets[j] + tensors[j]["bytes"])
+        offsets[i] = best[1] if best is not None else cursor
+        placed.append(i)
+    peak = max((offsets[i] + tensors[i]["bytes"] for i in range(n)), default=0)
+    return offsets, peak
+
+
+def overlapping_pairs(tensors, offsets):
+    """All pairs that are live together and share an address -- must be empty."""
+    bad = []
+    for i in range(len(tensors)):
+        for j in range(i + 1, len(tensors)):
+            if conflicts(tensors[i], tensors[j]):
+                a0, a1 = offsets[i], offsets[i] + tensors[i]["bytes"]
+                b0, b1 = offsets[j], offsets[j] + tensors[j]["bytes"]
+                if a0 < b1 and b0 < a1:
+                    bad.append((i, j))
+    return bad
+
+
+def chunks_for_budget(t, budget_bytes, max_chunks):
+    """Returns (chunks, peak) for the first C in 1..max_chunks whose arena peak fits,
+    or (None, smallest peak seen) when none does."""
+    smallest = None
+    for C in range(1, min(max_chunks, t.seq) + 1):
+        tensors, _ = _trace.trace(t, C)
+        _, peak = plan_arena(tensors)
+        if peak <= budget_bytes:
+            return C, peak
+        smallest = peak if smallest is None else min(smallest, peak)
+    return None, smallest

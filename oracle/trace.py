@@ -1,0 +1,109 @@
+"""Tensor-lifetime trace of the chunked DiT block template (test infrastructure only).
+
+The paper obtains lifetimes from one shape-only run of the pipeline and then
+treats them as template-static ("Offline Static Layout"; Memory Analyzer).
+There is no framework graph here, so the shape-only run is replaced by walking
+the block's own op list: every op names what it reads and writes, a tensor is
+born at the first op that writes it and dies after the last op that touches it
+(half-open lifetime [birth, death), as in Algorithm 1's input).
+
+Op order of one block with C sequence chunks (1 + 11 C ops):
+    MOD
+    for c: LN1A_c, KV_c, KROPE_c
+    for c: LN1B_c, Q_c, QROPE_c, ATTN_c, PROJ_c
+    for c: LN2_c, FFN1_c, FFN2_c
+Chunk c covers token rows [floor(c S / C), floor((c+1) S / C)).
+"""
+from __future__ import annotations
+
+ALIGN = 256
+
+KIND_INPUT, KIND_OUTPUT, KIND_FULL, KIND_CHUNK, KIND_WORKSPACE = range(5)
+DTYPE_BF16, DTYPE_F32 = 0, 1
+
+# row order of the tensor table; breaks ties between tensors born at the same op
+_ROW = {n: i for i, n in enumerate(
+    ("temb", "hid", "mod", "kv", "h1a", "h1b", "q", "o", "lse", "res", "h2", "g"))}
+
+
+def align_up(n, a=ALIGN):
+    return -(-n // a) * a
+
+
+def chunk_rows(S, C):
+    return [c * S // C for c in range(C + 1)]
+
+
+class _Recorder:
+    """Walks the op list; remembers first write and last touch of every tensor."""
+
+    def __init__(self):
+        self.t = 0
+        self.tensors = {}
+
+    def op(self, reads=(), writes=()):
+        for name in reads:
+            self.tensors[name]["death"] = self.t + 1
+        for name, meta in writes:
+            if name not in self.tensors:
+                self.tensors[name] = dict(meta, name=name, birth=self.t)
+            self.tensors[name]["death"] = self.t + 1
+        self.t += 1
+
+
+def trace(t, chunks):
+    """Returns (tensors, n_ops).  tensors: list of dicts with name, kind, dtype, block,
+    chunk, bytes (rounded up to 256), birth, death -- in id order (first birth, then
+    table row)."""
+    B, S, D, H, F, Dt = t.batch, t.seq, t.hidden, t.heads, t.ffn, t.temb_dim
+    C, L = chunks, t.n_blocks
+    if C < 1 or C > S:
+        raise ValueError("chunks must be in [1, S]")
+    r = chunk_rows(S, C)
+    rec = _Recorder()
+
+    def meta(base, nbytes, kind, dtype, block, chunk=-1):
+        return dict(base=base, bytes=align_up(nbytes), kind=kind, dtype=dtype, block=block, chunk=chunk)
+
+    u = 2 * B * S * D
+    # inputs exist before the first op
+    rec.tensors["temb"] = dict(meta("temb", 2 * B * Dt, KIND_INPUT, DTYPE_BF16, -1), name="temb", birth=0, death=1)
+    rec.tensors["hid0"] = dict(meta("hid", u, KIND_INPUT, DTYPE_BF16, 0), name="hid0", birth=0, death=1)
+    for l in range(L):
+        hid, nxt = f"hid{l}", f"hid{l + 1}"
+        mod, kv, res = f"mod{l}", f"kv{l}", f"res{l}"
+        m_mod = (mod, meta("mod", 24 * B * D, KIND_FULL, DTYPE_F32, l))
+        m_kv = (kv, meta("kv", 2 * u, KIND_FULL, DTYPE_BF16, l))
+        m_res = (res, meta("res", 2 * u, KIND_FULL, DTYPE_F32, l))
+        m_nxt = (nxt, meta("hid", u, KIND_OUTPUT if l + 1 == L else KIND_FULL, DTYPE_BF16, l + 1))
+        rec.op(reads=["temb"], writes=[m_mod])                                   # MOD
+        for c in range(C):
+            n = r[c + 1] - r[c]
+            h1a = (f"h1a{l}_{c}", meta("h1a", 2 * B * n * D, KIND_CHUNK, DTYPE_BF16, l, c))
+            rec.op(reads=[hid, mod], writes=[h1a])                               # LN1A
+            rec.op(reads=[h1a[0]], writes=[m_kv])                                # KV
+            rec.op(reads=[kv], writes=[m_kv])                                    # KROPE (in place)
+        for c in range(C):
+            n = r[c + 1] - r[c]
+            h1b = (f"h1b{l}_{c}", meta("h1b", 2 * B * n * D, KIND_CHUNK, DTYPE_BF16, l, c))
+            q = (f"q{l}_{c}", meta("q", 2 * B * n * D, KIND_CHUNK, DTYPE_BF16, l, c))
+            o = (f"o{l}_{c}", meta("o", 2 * B * n * D, KIND_CHUNK, DTYPE_BF16, l, c))
+            lse = (f"lse{l}_{c}", meta("lse", 4 * B * H * n, KIND_CHUNK, DTYPE_F32, l, c))
+            rec.op(reads=[hid, mod], writes=[h1b])                               # LN1B
+            rec.op(reads=[h1b[0]], writes=[q])                                   # Q
+            rec.op(reads=[q[0]], writes=[q])                                     # QROPE (in place)
+            rec.op(reads=[q[0], kv], writes=[o, lse])                            # ATTN
+            rec.op(reads=[o[0], hid, mod], writes=[m_res])                       # PROJ
+        for c in range(C):
+            n = r[c + 1] - r[c]
+            h2 = (f"h2{l}_{c}", meta("h2", 2 * B * n * D, KIND_CHUNK, DTYPE_BF16, l, c))
+            g = (f"g{l}_{c}", meta("g", 2 * B * n * F, KIND_CHUNK, DTYPE_BF16, l, c))
+            rec.op(reads=[res, mod], writes=[h2])                                # LN2
+            rec.op(reads=[h2[0]], writes=[g])                                    # FFN1
+            rec.op(reads=[g[0], res, mod], writes=[m_nxt])                       # FFN2
+    n_ops = rec.t
+    rec.tensors[f"hid{L}"]["death"] = n_ops          # the output outlives the last op
+    tensors = sorted(rec.tensors.values(), key=lambda d: (d["birth"], _ROW[d["base"]], d["chunk"]))
+    for d in tensors:
+        del d["base"]
+    return tensors, n_ops
