@@ -1,0 +1,246 @@
+/*
+ * xema.h -- C ABI of the B200 (sm_100a) library for memory-budgeted DiT blocks.
+ *
+ * The library implements the single-GPU hot path of Xema's fine-grained memory
+ * management for diffusion serving: a DiT denoising block (or a stack of blocks, one
+ * denoising step) is run sequence-chunked so that its activation peak fits a byte
+ * budget, and every intermediate tensor lives at a precomputed offset of one static
+ * arena derived from an offline lifetime trace instead of a caching allocator.
+ *
+ *   xema_trace              template + chunk count -> tensor sizes and lifetimes
+ *                           (the paper's Memory Analyzer; section "Memory Analysis and
+ *                           Latency Profiling" and "Offline Static Layout")
+ *   xema_plan_arena         lifetimes -> arena offsets (Algorithm 1, "Offline static
+ *                           memory layout") + reserved peak + max-live bytes
+ *   xema_chunks_for_budget  smallest chunk count whose reserved peak fits the budget
+ *                           (section "Applying Only as Much Mitigation as Needed", with the
+ *                           chunk count as the mitigation intensity; "Localized chunking")
+ *   xema_block_forward /    run one block / all n_blocks blocks on a caller-given CUDA
+ *   xema_step_forward       stream over caller-owned arena memory ("Static memory
+ *                           runtime": allocation at run time is a table lookup)
+ *
+ * Conventions
+ *   - All functions return 0 (XEMA_OK) or a negative xema_status; nothing throws, aborts,
+ *     allocates device memory, frees device memory or synchronises a stream or device.
+ *   - "host" / "device" is stated for every pointer.  Device pointers must belong to the
+ *     CUDA device that is current when the function is called.
+ *   - Linear layers are y = x W^T + b with W stored [out, in] row-major, bf16.
+ *   - Token rows: text tokens first, then the video/image tokens in (t, h, w) raster order.
+ *   - Chunk c of C covers token rows [floor(c*S/C), floor((c+1)*S/C)).
+ *   - Every tensor size is rounded up to 256 bytes, so every arena offset is 256-aligned.
+ */
+#ifndef XEMA_H_
+#define XEMA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum xema_status {
+  XEMA_OK = 0,
+  XEMA_EINVAL = -1,   /* bad argument or configuration                                   */
+  XEMA_ENOSPC = -2,   /* an output array or the arena is too small                        */
+  XEMA_EBUDGET = -3,  /* no chunk count up to max_chunks fits the budget                  */
+  XEMA_EALIGN = -4,   /* a device pointer is not aligned as required                      */
+  XEMA_ECUDA = -5,    /* a CUDA runtime/driver call failed; see xema_last_cuda_error()    */
+  XEMA_ETIMEOUT = -6, /* a kernel gave up a bounded wait (read back from the status word) */
+  XEMA_ESTATE = -7    /* the plan is not bound, or is bound for a different kind of call  */
+} xema_status;
+
+/* Request template.  Plain data, caller-owned, copied by the library. */
+typedef struct xema_config {
+  int32_t batch;      /* B >= 1; every chunk carries all B batch elements                 */
+  int32_t s_text;     /* text tokens (>= 0)                                               */
+  int32_t grid_t, grid_h, grid_w; /* latent grid; S = s_text + grid_t*grid_h*grid_w       */
+  int32_t hidden;     /* D = heads * head_dim; multiple of 256                            */
+  int32_t heads;      /* H                                                                */
+  int32_t head_dim;   /* dh: 64 or 128                                                    */
+  int32_t ffn;        /* F, multiple of 256                                               */
+  int32_t temb_dim;   /* Dt, multiple of 8                                                */
+  int32_t rope_dim_t, rope_dim_h, rope_dim_w; /* even, sum == head_dim                    */
+  float rope_base;    /* 10000                                                            */
+  float ln_eps;       /* LayerNorm epsilon (1e-6)                                         */
+  float rms_eps;      /* QK RMSNorm epsilon (1e-6)                                        */
+  int32_t n_blocks;   /* 1 = block template, 42 = CogVideoX-shaped denoising step         */
+} xema_config;
+
+enum { XEMA_KIND_INPUT = 0, XEMA_KIND_OUTPUT = 1, XEMA_KIND_FULL = 2, XEMA_KIND_CHUNK = 3,
+       XEMA_KIND_WORKSPACE = 4 };
+enum { XEMA_DTYPE_BF16 = 0, XEMA_DTYPE_F32 = 1 };
+
+/* One traced tensor.  Lifetime is the half-open interval [birth, death) of logical-op
+ * indices, as Algorithm 1 takes it. */
+typedef struct xema_tensor {
+  char name[24];   /* "hid0", "kv3", "q0_2", ... NUL-terminated                           */
+  uint32_t kind;   /* XEMA_KIND_*                                                         */
+  uint32_t dtype;  /* XEMA_DTYPE_*                                                        */
+  int32_t block;   /* block index, -1 for temb                                            */
+  int32_t chunk;   /* chunk index, -1 for full-sequence tensors                           */
+  uint64_t bytes;  /* rounded up to 256                                                   */
+  uint32_t birth;  /* first op that writes it (0 for inputs)                              */
+  uint32_t death;  /* 1 + last op that reads or writes it (n_ops for the output)          */
+} xema_tensor;
+
+/* Device pointers to one block's bf16 parameters. */
+typedef struct xema_block_weights {
+  const void* w_mod;  /* [6D, Dt]  adaLN modulation (shift1, scale1, gate1, shift2, ...)  */
+  const void* b_mod;  /* [6D]                                                             */
+  const void* w_qkv;  /* [3D, D]   rows 0..D-1 -> q, D..2D-1 -> k, 2D..3D-1 -> v          */
+  const void* b_qkv;  /* [3D]                                                             */
+  const void* g_q;    /* [dh]      RMSNorm gain of q                                      */
+  const void* g_k;    /* [dh]      RMSNorm gain of k                                      */
+  const void* w_o;    /* [D, D]                                                           */
+  const void* b_o;    /* [D]                                                              */
+  const void* w_1;    /* [F, D]                                                           */
+  const void* b_1;    /* [F]                                                              */
+  const void* w_2;    /* [D, F]                                                           */
+  const void* b_2;    /* [D]                                                              */
+} xema_block_weights;
+
+/* ---- host-only planner (pure integer code; no CUDA call) -------------------------------- */
+
+/* Tensor lifetimes of the template run with `chunks` sequence chunks (the offline,
+ * shape-only analysis of "Offline Static Layout").  Op order per block, 1 + 11*chunks ops:
+ * MOD; per chunk LN1A, KV, KROPE; per chunk LN1B, Q, QROPE, ATTN, PROJ; per chunk LN2,
+ * FFN1, FFN2.  Tensors are written to `out` (host, capacity `cap`) in id order = order of
+ * first birth.  *n_tensors (host) always receives the number of tensors, *n_ops (host) the
+ * number of ops, so a first call with cap = 0 sizes the array (returns XEMA_ENOSPC).
+ * XEMA_EINVAL: bad config or chunks outside [1, S]. */
+int xema_trace(const xema_config* cfg, int32_t chunks, xema_tensor* out, size_t cap,
+               size_t* n_tensors, uint32_t* n_ops);
+
+/* Algorithm 1 ("Offline static memory layout"): tensors in descending size (ties: birth,
+ * death, index); for each, the already placed tensors with an intersecting lifetime define
+ * address gaps; take the smallest gap that fits (ties: lowest address), else the address
+ * above all of them.  offsets (host, n entries) receives one byte offset per tensor;
+ * *peak_bytes = max(offset + bytes) is the reserved peak; *max_live_bytes is the largest sum
+ * of bytes live at one op (the active peak the reserved peak is compared with).  Either
+ * output pointer may be NULL. */
+int xema_plan_arena(const xema_tensor* tensors, size_t n, uint64_t* offsets,
+                    uint64_t* peak_bytes, uint64_t* max_live_bytes);
+
+/* Minimum mitigation that fits (section "Applying Only as Much Mitigation as Needed"):
+ * scans chunks = 1, 2, ..., max_chunks and returns the first whose reserved peak
+ * (xema_trace -> xema_plan_arena) is <= budget_bytes.  On XEMA_EBUDGET *chunks is 0 and
+ * *peak_bytes is the smallest peak seen. */
+int xema_chunks_for_budget(const xema_config* cfg, uint64_t budget_bytes, int32_t max_chunks,
+                           int32_t* chunks, uint64_t* peak_bytes);
+
+/* RoPE table for the template: host_out (host) receives S * (dh/2) * 2 floats laid out
+ * [token][pair][cos, sin]; angle = position * rope_base^(-2j/d) inside each of the three
+ * sections (t, h, w), evaluated in double precision and rounded once.  Text tokens sit at
+ * position (0, 0, 0).  The table is template-static parameter memory, not an arena tensor. */
+int xema_rope_table(const xema_config* cfg, float* host_out);
+
+/* ---- plan objects ----------------------------------------------------------------------- */
+
+typedef struct xema_plan xema_plan; /* opaque; host memory owned by the library */
+
+/* Traces and lays out the template for `chunks` chunks.  No CUDA call. */
+int xema_plan_create(const xema_config* cfg, int32_t chunks, xema_plan** out);
+void xema_plan_destroy(xema_plan* plan);
+
+/* Plan figures: any output pointer may be NULL. */
+int xema_plan_info(const xema_plan* plan, uint64_t* peak_bytes, uint64_t* max_live_bytes,
+                   size_t* n_tensors, uint32_t* n_ops, int32_t* chunks);
+/* Offset and (256-rounded) size of a tensor by name, e.g. "hid0", "temb", "hid1", "res0". */
+int xema_plan_tensor(const xema_plan* plan, const char* name, uint64_t* offset, uint64_t* bytes);
+/* Copy of the plan's tensor i and its offset. */
+int xema_plan_tensor_at(const xema_plan* plan, size_t i, xema_tensor* tensor, uint64_t* offset);
+
+/* Binds the plan to memory and pre-encodes every TMA descriptor (all addresses are static,
+ * so nothing is encoded at launch time).  arena_dev: device, 256-byte aligned, arena_bytes >=
+ * the plan's peak (XEMA_ENOSPC otherwise).  weights: host array of n_blocks structs holding
+ * device pointers (16-byte aligned).  rope_dev: device copy of xema_rope_table's output.
+ * status_dev: device, 4 bytes, zeroed by the caller, or NULL; kernels that give up a bounded
+ * wait store a non-zero code there.  Launches nothing.  The arena, weights and table stay
+ * owned by the caller and must outlive the forward calls. */
+int xema_plan_bind(xema_plan* plan, void* arena_dev, uint64_t arena_bytes,
+                   const xema_block_weights* weights, const float* rope_dev, void* status_dev);
+
+/* Enqueues the block (n_blocks must be 1) / all n_blocks blocks on `stream` (a cudaStream_t
+ * passed as void*).  Input: the caller has written hid0 [B,S,D] bf16 and temb [B,Dt] bf16 at
+ * their plan offsets; output: hid<n_blocks> [B,S,D] bf16 at its plan offset once the stream
+ * reaches the end of the enqueued work.  Every byte written lies inside [arena, arena+peak).
+ * Returns XEMA_ECUDA if a launch is rejected; asynchronous faults surface at the caller's
+ * own synchronisation. */
+int xema_block_forward(const xema_plan* plan, void* stream);
+int xema_step_forward(const xema_plan* plan, void* stream);
+
+/* Number of kernel launches one forward call enqueues (0 if unbound). */
+int xema_plan_launch_count(const xema_plan* plan);
+
+/* Debug aid: enqueue only the first n_logical_ops logical ops of the trace order. */
+int xema_forward_prefix(const xema_plan* plan, uint32_t n_logical_ops, void* stream);
+
+/* ---- single operators (the kernels behind the forward calls, on plain device pointers) --- */
+
+/* mod[b, j] = sum_k silu(temb[b,k]) w_mod[j,k] + b_mod[j]; temb [B,Dt] bf16, w_mod [n_out,Dt]
+ * bf16, b_mod [n_out] bf16 -> mod [B,n_out] fp32 (all device). */
+int xema_op_mod(const void* temb, const void* w_mod, const void* b_mod, float* mod, int32_t batch,
+                int32_t temb_dim, int32_t n_out, void* stream);
+
+/* out[b,i,:] = LN(in[b,i,:]) * (1 + scale[b,:]) + shift[b,:]; LayerNorm without affine,
+ * biased variance.  in: device, bf16 (in_is_f32 = 0) or fp32 (1), row (b,i) at element
+ * (b*in_batch_rows + i)*D; out: device bf16 [B,rows,D] contiguous; shift/scale: device fp32,
+ * batch stride mod_stride elements. */
+int xema_op_ln_modulate(const void* in, int32_t in_is_f32, int64_t in_batch_rows, void* out,
+                        const float* shift, const float* scale, int64_t mod_stride, int32_t batch,
+                        int32_t rows, int32_t D, float eps, void* stream);
+
+/* In place, per head: x <- RoPE(x / sqrt(mean(x^2) + eps) * g).  x: device bf16, row (b,i) at
+ * element (b*batch_rows + i)*ld, heads*head_dim leading features of each row are touched.
+ * rope: device fp32 [*, head_dim/2, 2] indexed by token = pos0 + i.  g: device bf16 [head_dim]. */
+int xema_op_rmsnorm_rope(void* x, int64_t ld, int64_t batch_rows, const void* g, const float* rope,
+                         int32_t pos0, int32_t batch, int32_t rows, int32_t heads, int32_t head_dim,
+                         float eps, void* stream);
+
+/* Epilogues of the tensor-core GEMM acc = A[b] (rows x K) * W^T (N x K), fp32 accumulate. */
+enum {
+  XEMA_EPI_BIAS = 0,       /* out bf16 = acc + bias                                        */
+  XEMA_EPI_BIAS_GELU = 1,  /* out bf16 = gelu_tanh(acc + bias)                             */
+  XEMA_EPI_GATE_RES_F32 = 2,  /* out fp32 = resid(bf16) + gate[b,:] * (acc + bias)         */
+  XEMA_EPI_GATE_RES_BF16 = 3  /* out bf16 = resid(fp32) + gate[b,:] * (acc + bias)         */
+};
+typedef struct xema_gemm_args {
+  const void* a;        /* device bf16, row (b,i) at element (b*a_batch_rows + i)*lda      */
+  int64_t lda, a_batch_rows;
+  const void* w;        /* device bf16 [N, K], row stride ldw                              */
+  int64_t ldw;
+  const void* bias;     /* device bf16 [N]                                                 */
+  void* out;            /* device, row (b,i) at element (b*out_batch_rows + i)*ldo         */
+  int64_t ldo, out_batch_rows;
+  const void* resid;    /* device, same row addressing with ldr / resid_batch_rows; or NULL */
+  int64_t ldr, resid_batch_rows;
+  const float* gate;    /* device fp32, gate[b*gate_stride + n]; or NULL                   */
+  int64_t gate_stride;
+  int32_t batch, rows, N, K; /* N % 128 == 0, K % 64 == 0                                  */
+  int32_t epilogue;     /* XEMA_EPI_*                                                      */
+} xema_gemm_args;
+int xema_op_gemm(const xema_gemm_args* args, void* status_dev, void* stream);
+
+/* Non-causal attention of `rows` query rows against all `keys` keys, per (batch, head):
+ * o = softmax(q k^T / sqrt(head_dim)) v, lse = log sum exp (natural log).
+ * q: device bf16, row (b,i) at (b*q_batch_rows + i)*ldq, head h at feature h*head_dim.
+ * k, v: device bf16, key (b,j) at (b*kv_batch_rows + j)*ldkv (k and v are separate base
+ * pointers into the same rows).  o: device bf16 [B,rows,heads*head_dim] contiguous.
+ * lse: device fp32 [B,heads,rows] or NULL. */
+int xema_op_attention(const void* q, int64_t ldq, int64_t q_batch_rows, const void* k, const void* v,
+                      int64_t ldkv, int64_t kv_batch_rows, void* o, float* lse, int32_t batch,
+                      int32_t rows, int32_t keys, int32_t heads, int32_t head_dim, void* status_dev,
+                      void* stream);
+
+/* ---- diagnostics ------------------------------------------------------------------------ */
+const char* xema_strerror(int status);
+/* Last cudaError_t / CUresult seen by this thread's most recent failing call (0 if none). */
+int xema_last_cuda_error(void);
+/* Library version string, e.g. "xema-b200 0.1 (sm_100a)". */
+const char* xema_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* XEMA_H_ */

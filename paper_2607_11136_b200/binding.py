@@ -1,0 +1,273 @@
+"""ctypes binding of libxema.so: the same names as the C ABI, argument marshalling only.
+
+Every step of the hot path runs inside the CUDA library.  There is no CPU fallback: if the
+library is missing, loading raises, and nothing here imports the test oracle.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libxema.so")
+
+XEMA_OK, XEMA_EINVAL, XEMA_ENOSPC, XEMA_EBUDGET = 0, -1, -2, -3
+XEMA_EALIGN, XEMA_ECUDA, XEMA_ETIMEOUT, XEMA_ESTATE = -4, -5, -6, -7
+EPI_BIAS, EPI_BIAS_GELU, EPI_GATE_RES_F32, EPI_GATE_RES_BF16 = 0, 1, 2, 3
+
+EXPORTS = (
+    "xema_trace", "xema_plan_arena", "xema_chunks_for_budget", "xema_rope_table",
+    "xema_plan_create", "xema_plan_destroy", "xema_plan_info", "xema_plan_tensor",
+    "xema_plan_tensor_at", "xema_plan_bind", "xema_block_forward", "xema_step_forward",
+    "xema_plan_launch_count", "xema_forward_prefix", "xema_op_mod", "xema_op_ln_modulate",
+    "xema_op_rmsnorm_rope", "xema_op_gemm", "xema_op_attention", "xema_strerror",
+    "xema_last_cuda_error", "xema_version",
+)
+
+
+class XemaError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = "%s: %s (status %d" % (where, strerror(status), status)
+        if status == XEMA_ECUDA:
+            msg += ", cuda error %d" % last_cuda_error()
+        super().__init__(msg + ")")
+
+
+class xema_config(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("batch", "s_text", "grid_t", "grid_h", "grid_w", "hidden", "heads",
+                                         "head_dim", "ffn", "temb_dim", "rope_dim_t", "rope_dim_h", "rope_dim_w")]
+    _fields_ += [("rope_base", C.c_float), ("ln_eps", C.c_float), ("rms_eps", C.c_float), ("n_blocks", C.c_int32)]
+
+
+class xema_tensor(C.Structure):
+    _fields_ = [("name", C.c_char * 24), ("kind", C.c_uint32), ("dtype", C.c_uint32), ("block", C.c_int32),
+                ("chunk", C.c_int32), ("bytes", C.c_uint64), ("birth", C.c_uint32), ("death", C.c_uint32)]
+
+
+_WEIGHT_FIELDS = ("w_mod", "b_mod", "w_qkv", "b_qkv", "g_q", "g_k", "w_o", "b_o", "w_1", "b_1", "w_2", "b_2")
+
+
+class xema_block_weights(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in _WEIGHT_FIELDS]
+
+
+class xema_gemm_args(C.Structure):
+    _fields_ = [("a", C.c_void_p), ("lda", C.c_int64), ("a_batch_rows", C.c_int64),
+                ("w", C.c_void_p), ("ldw", C.c_int64), ("bias", C.c_void_p),
+                ("out", C.c_void_p), ("ldo", C.c_int64), ("out_batch_rows", C.c_int64),
+                ("resid", C.c_void_p), ("ldr", C.c_int64), ("resid_batch_rows", C.c_int64),
+                ("gate", C.c_void_p), ("gate_stride", C.c_int64),
+                ("batch", C.c_int32), ("rows", C.c_int32), ("N", C.c_int32), ("K", C.c_int32),
+                ("epilogue", C.c_int32)]
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Loads libxema.so (built in-tree by paper_2607_11136_b200.build).  Raises if it is absent."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError("libxema.so is not built: run `python -m paper_2607_11136_b200.build` "
+                              "(there is no CPU fallback)")
+        L = C.CDLL(LIB_PATH)
+        vp, i32, i64, u64, u32, sz = C.c_void_p, C.c_int32, C.c_int64, C.c_uint64, C.c_uint32, C.c_size_t
+        P = C.POINTER
+        sig = {
+            "xema_trace": [P(xema_config), i32, P(xema_tensor), sz, P(sz), P(u32)],
+            "xema_plan_arena": [P(xema_tensor), sz, P(u64), P(u64), P(u64)],
+            "xema_chunks_for_budget": [P(xema_config), u64, i32, P(i32), P(u64)],
+            "xema_rope_table": [P(xema_config), vp],
+            "xema_plan_create": [P(xema_config), i32, P(vp)],
+            "xema_plan_info": [vp, P(u64), P(u64), P(sz), P(u32), P(i32)],
+            "xema_plan_tensor": [vp, C.c_char_p, P(u64), P(u64)],
+            "xema_plan_tensor_at": [vp, sz, P(xema_tensor), P(u64)],
+            "xema_plan_bind": [vp, vp, u64, P(xema_block_weights), vp, vp],
+            "xema_block_forward": [vp, vp],
+            "xema_step_forward": [vp, vp],
+            "xema_plan_launch_count": [vp],
+            "xema_forward_prefix": [vp, u32, vp],
+            "xema_op_mod": [vp, vp, vp, vp, i32, i32, i32, vp],
+            "xema_op_ln_modulate": [vp, i32, i64, vp, vp, vp, i64, i32, i32, i32, C.c_float, vp],
+            "xema_op_rmsnorm_rope": [vp, i64, i64, vp, vp, i32, i32, i32, i32, i32, C.c_float, vp],
+            "xema_op_gemm": [P(xema_gemm_args), vp, vp],
+            "xema_op_attention": [vp, i64, i64, vp, vp, i64, i64, vp, vp, i32, i32, i32, i32, i32, vp, vp],
+            "xema_last_cuda_error": [],
+        }
+        for name, args in sig.items():
+            fn = getattr(L, name)
+            fn.argtypes = args
+            fn.restype = C.c_int
+        L.xema_plan_destroy.argtypes = [vp]
+        L.xema_plan_destroy.restype = None
+        L.xema_strerror.argtypes = [C.c_int]
+        L.xema_strerror.restype = C.c_char_p
+        L.xema_version.argtypes = []
+        L.xema_version.restype = C.c_char_p
+        _lib = L
+    return _lib
+
+
+def _check(status: int, where: str) -> None:
+    if status != XEMA_OK:
+        raise XemaError(status, where)
+
+
+def strerror(status: int) -> str:
+    return lib().xema_strerror(status).decode()
+
+
+def last_cuda_error() -> int:
+    return lib().xema_last_cuda_error()
+
+
+def version() -> str:
+    return lib().xema_version().decode()
+
+
+def make_config(t) -> xema_config:
+    """xema_config from any object with the template's attribute names."""
+    c = xema_config()
+    for name, _ in xema_config._fields_:
+        setattr(c, name, getattr(t, name))
+    return c
+
+
+def _tensor_dict(t: xema_tensor) -> dict:
+    return {"name": t.name.decode(), "kind": t.kind, "dtype": t.dtype, "block": t.block, "chunk": t.chunk,
+            "bytes": t.bytes, "birth": t.birth, "death": t.death}
+
+
+def xema_trace(cfg: xema_config, chunks: int):
+    """-> (list of tensor dicts in id order, n_ops)"""
+    n, ops = C.c_size_t(0), C.c_uint32(0)
+    rc = lib().xema_trace(C.byref(cfg), chunks, None, 0, C.byref(n), C.byref(ops))
+    if rc != XEMA_ENOSPC:
+        _check(rc, "xema_trace")
+    arr = (xema_tensor * n.value)()
+    _check(lib().xema_trace(C.byref(cfg), chunks, arr, n.value, C.byref(n), C.byref(ops)), "xema_trace")
+    return [_tensor_dict(t) for t in arr], ops.value
+
+
+def xema_plan_arena(tensors: Sequence[dict]):
+    """tensors: dicts with bytes, birth, death -> (offsets, peak_bytes, max_live_bytes)"""
+    n = len(tensors)
+    arr = (xema_tensor * max(n, 1))()
+    for i, d in enumerate(tensors):
+        arr[i].bytes, arr[i].birth, arr[i].death = d["bytes"], d["birth"], d["death"]
+    offs = (C.c_uint64 * max(n, 1))()
+    peak, live = C.c_uint64(0), C.c_uint64(0)
+    _check(lib().xema_plan_arena(arr, n, offs, C.byref(peak), C.byref(live)), "xema_plan_arena")
+    return list(offs[:n]), peak.value, live.value
+
+
+def xema_chunks_for_budget(cfg: xema_config, budget_bytes: int, max_chunks: int):
+    """-> (chunks, peak_bytes); chunks is None when nothing fits (peak = smallest seen)."""
+    ch, peak = C.c_int32(0), C.c_uint64(0)
+    rc = lib().xema_chunks_for_budget(C.byref(cfg), budget_bytes, max_chunks, C.byref(ch), C.byref(peak))
+    if rc == XEMA_EBUDGET:
+        return None, peak.value
+    _check(rc, "xema_chunks_for_budget")
+    return ch.value, peak.value
+
+
+def xema_rope_table(cfg: xema_config) -> np.ndarray:
+    S = cfg.s_text + cfg.grid_t * cfg.grid_h * cfg.grid_w
+    out = np.empty((S, cfg.head_dim // 2, 2), dtype=np.float32)
+    _check(lib().xema_rope_table(C.byref(cfg), out.ctypes.data_as(C.c_void_p)), "xema_rope_table")
+    return out
+
+
+class Plan:
+    """Owner of an xema_plan handle."""
+
+    def __init__(self, cfg: xema_config, chunks: int):
+        self.cfg = cfg
+        self._h = C.c_void_p()
+        _check(lib().xema_plan_create(C.byref(cfg), chunks, C.byref(self._h)), "xema_plan_create")
+        peak, live, n, ops, ch = C.c_uint64(), C.c_uint64(), C.c_size_t(), C.c_uint32(), C.c_int32()
+        _check(lib().xema_plan_info(self._h, C.byref(peak), C.byref(live), C.byref(n), C.byref(ops), C.byref(ch)),
+               "xema_plan_info")
+        self.peak_bytes, self.max_live_bytes = peak.value, live.value
+        self.n_tensors, self.n_ops, self.chunks = n.value, ops.value, ch.value
+        self._keep = None
+
+    def close(self):
+        if self._h:
+            lib().xema_plan_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def tensor(self, name: str):
+        off, nbytes = C.c_uint64(), C.c_uint64()
+        _check(lib().xema_plan_tensor(self._h, name.encode(), C.byref(off), C.byref(nbytes)), "xema_plan_tensor")
+        return off.value, nbytes.value
+
+    def tensors(self):
+        out = []
+        for i in range(self.n_tensors):
+            t, off = xema_tensor(), C.c_uint64()
+            _check(lib().xema_plan_tensor_at(self._h, i, C.byref(t), C.byref(off)), "xema_plan_tensor_at")
+            d = _tensor_dict(t)
+            d["offset"] = off.value
+            out.append(d)
+        return out
+
+    def bind(self, arena_ptr: int, arena_bytes: int, weights: Sequence[dict], rope_ptr: int,
+             status_ptr: Optional[int] = None):
+        """weights: one dict per block mapping the twelve parameter names to device pointers."""
+        arr = (xema_block_weights * len(weights))()
+        for i, w in enumerate(weights):
+            for f in _WEIGHT_FIELDS:
+                setattr(arr[i], f, w[f])
+        _check(lib().xema_plan_bind(self._h, arena_ptr, arena_bytes, arr, rope_ptr, status_ptr), "xema_plan_bind")
+        self._keep = arr
+
+    def launch_count(self) -> int:
+        return lib().xema_plan_launch_count(self._h)
+
+    def block_forward(self, stream: int = 0):
+        _check(lib().xema_block_forward(self._h, stream), "xema_block_forward")
+
+    def step_forward(self, stream: int = 0):
+        _check(lib().xema_step_forward(self._h, stream), "xema_step_forward")
+
+    def forward_prefix(self, n_logical_ops: int, stream: int = 0):
+        _check(lib().xema_forward_prefix(self._h, n_logical_ops, stream), "xema_forward_prefix")
+
+
+def xema_op_mod(temb, w_mod, b_mod, mod, batch, temb_dim, n_out, stream=0):
+    _check(lib().xema_op_mod(temb, w_mod, b_mod, mod, batch, temb_dim, n_out, stream), "xema_op_mod")
+
+
+def xema_op_ln_modulate(inp, in_is_f32, in_batch_rows, out, shift, scale, mod_stride, batch, rows, D, eps, stream=0):
+    _check(lib().xema_op_ln_modulate(inp, in_is_f32, in_batch_rows, out, shift, scale, mod_stride, batch, rows, D,
+                                     eps, stream), "xema_op_ln_modulate")
+
+
+def xema_op_rmsnorm_rope(x, ld, batch_rows, g, rope, pos0, batch, rows, heads, head_dim, eps, stream=0):
+    _check(lib().xema_op_rmsnorm_rope(x, ld, batch_rows, g, rope, pos0, batch, rows, heads, head_dim, eps, stream),
+           "xema_op_rmsnorm_rope")
+
+
+def xema_op_gemm(status=None, stream=0, **kw):
+    a = xema_gemm_args()
+    for k, v in kw.items():
+        setattr(a, k, v)
+    _check(lib().xema_op_gemm(C.byref(a), status, stream), "xema_op_gemm")
+
+
+def xema_op_attention(q, ldq, q_batch_rows, k, v, ldkv, kv_batch_rows, o, lse, batch, rows, keys, heads, head_dim,
+                      status=None, stream=0):
+    _check(lib().xema_op_attention(q, ldq, q_batch_rows, k, v, ldkv, kv_batch_rows, o, lse, batch, rows, keys, heads,
+                                   head_dim, status, stream), "xema_op_attention")

@@ -1,0 +1,374 @@
+// Non-causal flash-style attention on tcgen05: o = softmax(q k^T / sqrt(dh)) v over all keys.
+//
+// One CTA owns one (batch, head, 128-query-row tile) and streams the keys in blocks of 128;
+// its workspace (shared memory and TMEM) depends on the query tile only, never on the number
+// of keys.  192 threads:
+//   warp 0    TMA producer: Q tile once, then K and V tiles through two-stage rings
+//   warp 1    owns TMEM; one thread issues S = Q K^T (TMEM, 128 fp32 columns) and
+//             O += P V (TMEM, dh fp32 columns)
+//   warps 2-5 softmax: thread = query row.  Read S from TMEM, running max / sum in the exp2
+//             domain, write P (bf16) into shared memory in the 128-byte-swizzled K-major
+//             layout the MMA reads, rescale O in TMEM when the running max moved, and at
+//             the end normalise O and store it.
+// Every decision is taken per row (the running max only moves when it grows by more than 2^8
+// in the exp2 domain; multiplying the other rows by exactly 1 changes nothing), keys are
+// always visited from key 0 in blocks of 128, and nothing is split or reduced across CTAs, so
+// a query row's output bits do not depend on how the query rows are chunked or tiled.
+#include <algorithm>
+
+#include "kernels.h"
+#include "sm100.cuh"
+
+namespace xema {
+using namespace sm100;
+
+constexpr int ATT_BM = 128;      // query rows per CTA
+constexpr int ATT_BN = 128;      // keys per block
+constexpr int ATT_THREADS = 192;
+constexpr int ATT_KV_STAGES = 2;
+constexpr int ATOM_BYTES = 128 * 128;   // 128 rows x 64 bf16, one swizzled column block
+
+template <int DH>
+struct AttnCfg {
+  static constexpr int ATOMS = DH / 64;                      // 64-wide column blocks per tile
+  static constexpr int TILE_BYTES = ATOMS * ATOM_BYTES;      // Q, K or V tile
+  static constexpr int P_BYTES = (ATT_BN / 64) * ATOM_BYTES;
+  static constexpr int OFF_Q = 0;
+  static constexpr int OFF_K = OFF_Q + TILE_BYTES;
+  static constexpr int OFF_V = OFF_K + ATT_KV_STAGES * TILE_BYTES;
+  static constexpr int OFF_P = OFF_V + ATT_KV_STAGES * TILE_BYTES;
+  static constexpr int OFF_BAR = OFF_P + P_BYTES;
+  static constexpr int SMEM_BYTES = OFF_BAR + 256;
+  static constexpr int TMEM_COLS = 256;                      // S: [0,128), O: [128, 128+DH)
+  static constexpr int TMEM_O = 128;
+  static constexpr int MIN_CTAS = (DH == 64) ? 2 : 1;
+};
+
+struct AttnParams {
+  __nv_bfloat16* o;
+  float* lse;
+  int batch, rows, keys, heads;
+  float scale;        // 1/sqrt(dh)
+  float scale_log2;   // scale * log2(e)
+  unsigned int* status;
+};
+
+template <int DH>
+__global__ void __launch_bounds__(ATT_THREADS, AttnCfg<DH>::MIN_CTAS)
+attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                 const __grid_constant__ CUtensorMap map_v, const AttnParams p) {
+  using Cfg = AttnCfg<DH>;
+  extern __shared__ __align__(1024) uint8_t smem[];
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + Cfg::OFF_BAR);
+  uint64_t* q_full = bars + 0;
+  uint64_t* k_full = bars + 1;    // [2]
+  uint64_t* k_empty = bars + 3;   // [2]
+  uint64_t* v_full = bars + 5;    // [2]
+  uint64_t* v_empty = bars + 7;   // [2]
+  uint64_t* s_full = bars + 9;
+  uint64_t* p_full = bars + 10;
+  uint64_t* pv_done = bars + 11;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 12);
+  volatile uint32_t* abort_flag = tmem_slot + 1;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int qt = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+  const int n_kv = (p.keys + ATT_BN - 1) / ATT_BN;
+
+  // The swizzled tiles need a 1024-byte aligned base; refuse to run otherwise.
+  if ((smem_u32(smem) & 1023u) != 0) {
+    if (threadIdx.x == 0 && p.status) atomicExch(p.status, 0x54310002u);
+    return;
+  }
+
+  if (threadIdx.x == 0) {
+    mbar_init(q_full, 1);
+    for (int s = 0; s < ATT_KV_STAGES; ++s) {
+      mbar_init(&k_full[s], 1);
+      mbar_init(&k_empty[s], 1);
+      mbar_init(&v_full[s], 1);
+      mbar_init(&v_empty[s], 1);
+    }
+    mbar_init(s_full, 1);
+    mbar_init(p_full, 4);
+    mbar_init(pv_done, 1);
+    *abort_flag = 0;
+    fence_mbar_init();
+    prefetch_tmap(&map_q);
+    prefetch_tmap(&map_k);
+    prefetch_tmap(&map_v);
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_slot, Cfg::TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t tmem_s = tmem_base;
+  const uint32_t tmem_o = tmem_base + Cfg::TMEM_O;
+
+  if (warp == 0) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0) {
+      bool ok = true;
+      mbar_expect_tx(q_full, Cfg::TILE_BYTES);
+#pragma unroll
+      for (int a = 0; a < Cfg::ATOMS; ++a)
+        tma_load_3d(smem + Cfg::OFF_Q + a * ATOM_BYTES, &map_q, q_full, h * DH + a * 64, qt * ATT_BM, b);
+      int k_issued = 0, v_issued = 0;
+      for (int j = 0; j < n_kv; ++j) {
+        const int st = j % ATT_KV_STAGES;
+        const uint32_t ph = (uint32_t)(j / ATT_KV_STAGES) & 1u;
+        if (!(ok = mbar_wait(&k_empty[st], ph ^ 1, abort_flag))) break;
+        mbar_expect_tx(&k_full[st], Cfg::TILE_BYTES);
+#pragma unroll
+        for (int a = 0; a < Cfg::ATOMS; ++a)
+          tma_load_3d(smem + Cfg::OFF_K + st * Cfg::TILE_BYTES + a * ATOM_BYTES, &map_k, &k_full[st],
+                      h * DH + a * 64, j * ATT_BN, b);
+        k_issued = j + 1;
+        if (!(ok = mbar_wait(&v_empty[st], ph ^ 1, abort_flag))) break;
+        mbar_expect_tx(&v_full[st], Cfg::TILE_BYTES);
+#pragma unroll
+        for (int a = 0; a < Cfg::ATOMS; ++a)
+          tma_load_3d(smem + Cfg::OFF_V + st * Cfg::TILE_BYTES + a * ATOM_BYTES, &map_v, &v_full[st],
+                      h * DH + a * 64, j * ATT_BN, b);
+        v_issued = j + 1;
+      }
+      if (!ok) {
+        // gave up: let the copies already issued land before the CTA leaves (the latest
+        // fill of each stage; older fills were consumed before their stage was reused)
+        volatile uint32_t dummy = 0;
+        mbar_wait(q_full, 0, &dummy);
+        for (int j = max(0, k_issued - ATT_KV_STAGES); j < k_issued; ++j) {
+          dummy = 0;
+          mbar_wait(&k_full[j % ATT_KV_STAGES], (uint32_t)(j / ATT_KV_STAGES) & 1u, &dummy);
+        }
+        for (int j = max(0, v_issued - ATT_KV_STAGES); j < v_issued; ++j) {
+          dummy = 0;
+          mbar_wait(&v_full[j % ATT_KV_STAGES], (uint32_t)(j / ATT_KV_STAGES) & 1u, &dummy);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      constexpr uint32_t idesc_s = idesc_bf16_f32(ATT_BM, ATT_BN, false, false);   // S = Q K^T
+      constexpr uint32_t idesc_o = idesc_bf16_f32(ATT_BM, DH, false, true);        // O = P V, V is N-major
+      const uint32_t q_addr = smem_u32(smem + Cfg::OFF_Q);
+      const uint32_t p_addr = smem_u32(smem + Cfg::OFF_P);
+      auto issue_s = [&](int j) -> bool {
+        const int st = j % ATT_KV_STAGES;
+        const uint32_t ph = (uint32_t)(j / ATT_KV_STAGES) & 1u;
+        if (!mbar_wait(&k_full[st], ph, abort_flag)) return false;
+        tc_fence_after();
+        const uint32_t k_addr = smem_u32(smem + Cfg::OFF_K + st * Cfg::TILE_BYTES);
+#pragma unroll
+        for (int k = 0; k < DH / 16; ++k) {
+          const uint32_t off = (k / 4) * ATOM_BYTES + (k % 4) * 32;
+          mma_ss(tmem_s, smem_desc_sw128(q_addr + off, 16, 1024), smem_desc_sw128(k_addr + off, 16, 1024), idesc_s,
+                 k != 0);
+        }
+        mma_commit(&k_empty[st]);
+        mma_commit(s_full);
+        return true;
+      };
+      bool ok = mbar_wait(q_full, 0, abort_flag);
+      if (ok) ok = issue_s(0);
+      for (int j = 0; ok && j < n_kv; ++j) {
+        const int st = j % ATT_KV_STAGES;
+        const uint32_t ph = (uint32_t)(j / ATT_KV_STAGES) & 1u;
+        // softmax has read all of S(j) and written P(j)
+        if (!(ok = mbar_wait(p_full, j & 1, abort_flag))) break;
+        tc_fence_after();
+        if (j + 1 < n_kv && !(ok = issue_s(j + 1))) break;
+        if (!(ok = mbar_wait(&v_full[st], ph, abort_flag))) break;
+        tc_fence_after();
+        const uint32_t v_addr = smem_u32(smem + Cfg::OFF_V + st * Cfg::TILE_BYTES);
+#pragma unroll
+        for (int kk = 0; kk < ATT_BN / 16; ++kk) {
+          const uint64_t da = smem_desc_sw128(p_addr + (kk / 4) * ATOM_BYTES + (kk % 4) * 32, 16, 1024);
+          // V tile: rows = keys (the MMA's K), 64 dh per 128-byte row; 16 keys = 2048 bytes;
+          // the second 64-wide dh block (dh = 128) starts one atom further
+          const uint64_t db = smem_desc_sw128(v_addr + kk * 2048, ATOM_BYTES, 1024);
+          mma_ss(tmem_o, da, db, idesc_o, (j | kk) != 0);
+        }
+        mma_commit(&v_empty[st]);
+        mma_commit(pv_done);
+      }
+    }
+  } else {
+    // ---------------- softmax / correction / epilogue ----------------
+    const int quad = warp & 3;
+    const int r = quad * 32 + lane;                       // query row inside the tile = TMEM lane
+    const uint32_t lane_sel = (uint32_t)(quad * 32) << 16;
+    uint8_t* p_row = smem + Cfg::OFF_P + r * 128;
+    const int swz = r & 7;
+    float m_run = -INFINITY, l_run = 0.f;
+    bool ok = true;
+    for (int j = 0; j < n_kv; ++j) {
+      ok = mbar_wait(s_full, j & 1, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      const int valid = min(ATT_BN, p.keys - j * ATT_BN);   // < 128 only in the last block
+      // pass 1: row max of the raw scores
+      float m_blk = -INFINITY;
+#pragma unroll 1
+      for (int ch = 0; ch < ATT_BN / 32; ++ch) {
+        uint32_t s[32];
+        tmem_ld32(tmem_s + lane_sel + ch * 32, s);
+        tmem_ld_wait();
+#pragma unroll
+        for (int t = 0; t < 32; ++t) {
+          const float v = (ch * 32 + t < valid) ? __uint_as_float(s[t]) : -INFINITY;
+          m_blk = fmaxf(m_blk, v);
+        }
+      }
+      // the running max moves only when it grows by more than 2^8 (exp2 domain); per row
+      float m_new = m_run;
+      if (j == 0 || (m_blk - m_run) * p.scale_log2 > 8.f) m_new = m_blk;
+      const float alpha = (j == 0 || m_new == m_run) ? 1.f : ex2_approx((m_run - m_new) * p.scale_log2);
+      const float neg_m = -m_new * p.scale_log2;
+      // P(j) overwrites the buffer PV(j-1) reads, and O must be at rest before it is rescaled
+      if (j > 0) {
+        ok = mbar_wait(pv_done, (j - 1) & 1, abort_flag);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after();
+      }
+      // pass 2: p = exp2(s * c - m * c), row sum, bf16 P into swizzled shared memory
+      float l_blk = 0.f;
+#pragma unroll 1
+      for (int ch = 0; ch < ATT_BN / 32; ++ch) {
+        uint32_t s[32];
+        tmem_ld32(tmem_s + lane_sel + ch * 32, s);
+        tmem_ld_wait();
+        float pv[32];
+#pragma unroll
+        for (int t = 0; t < 32; ++t) {
+          const float e = ex2_approx(fmaf(__uint_as_float(s[t]), p.scale_log2, neg_m));
+          pv[t] = (ch * 32 + t < valid) ? e : 0.f;
+          l_blk += pv[t];
+        }
+        uint8_t* atom_row = p_row + (ch / 2) * ATOM_BYTES;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const int chunk16 = (ch & 1) * 4 + q;             // 16-byte chunk inside the 128-byte row
+          uint4 w = make_uint4(pack_bf16x2(pv[8 * q + 0], pv[8 * q + 1]), pack_bf16x2(pv[8 * q + 2], pv[8 * q + 3]),
+                               pack_bf16x2(pv[8 * q + 4], pv[8 * q + 5]), pack_bf16x2(pv[8 * q + 6], pv[8 * q + 7]));
+          *reinterpret_cast<uint4*>(atom_row + ((chunk16 ^ swz) << 4)) = w;
+        }
+      }
+      l_run = fmaf(l_run, alpha, l_blk);
+      m_run = m_new;
+      // rescale O where the max moved (rows that kept their max multiply by exactly 1)
+      if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+#pragma unroll 1
+        for (int ch = 0; ch < DH / 32; ++ch) {
+          uint32_t o[32];
+          tmem_ld32(tmem_o + lane_sel + ch * 32, o);
+          tmem_ld_wait();
+#pragma unroll
+          for (int t = 0; t < 32; ++t) o[t] = __float_as_uint(__uint_as_float(o[t]) * alpha);
+          tmem_st32(tmem_o + lane_sel + ch * 32, o);
+        }
+        tmem_st_wait();
+      }
+      fence_proxy_async_smem();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(p_full);
+    }
+    if (ok) {
+      ok = mbar_wait(pv_done, (n_kv - 1) & 1, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+    }
+    if (ok) {
+      tc_fence_after();
+      const int row = qt * ATT_BM + r;
+      const float inv_l = 1.f / l_run;
+      __nv_bfloat16* orow = p.o + ((size_t)b * p.rows + row) * ((size_t)p.heads * DH) + (size_t)h * DH;
+#pragma unroll 1
+      for (int ch = 0; ch < DH / 32; ++ch) {
+        uint32_t o[32];
+        tmem_ld32(tmem_o + lane_sel + ch * 32, o);
+        tmem_ld_wait();
+        if (row < p.rows) {
+          uint4* dst = reinterpret_cast<uint4*>(orow + ch * 32);
+#pragma unroll
+          for (int q = 0; q < 4; ++q)
+            dst[q] = make_uint4(pack_bf16x2(__uint_as_float(o[8 * q + 0]) * inv_l, __uint_as_float(o[8 * q + 1]) * inv_l),
+                                pack_bf16x2(__uint_as_float(o[8 * q + 2]) * inv_l, __uint_as_float(o[8 * q + 3]) * inv_l),
+                                pack_bf16x2(__uint_as_float(o[8 * q + 4]) * inv_l, __uint_as_float(o[8 * q + 5]) * inv_l),
+                                pack_bf16x2(__uint_as_float(o[8 * q + 6]) * inv_l, __uint_as_float(o[8 * q + 7]) * inv_l));
+        }
+      }
+      if (p.lse && row < p.rows)
+        p.lse[((size_t)b * p.heads + h) * p.rows + row] = fmaf(m_run, p.scale, logf(l_run));
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, Cfg::TMEM_COLS);
+  }
+  if (threadIdx.x == 0 && *abort_flag && p.status) atomicExch(p.status, STATUS_TIMEOUT_MBARRIER);
+}
+
+template <int DH>
+static int launch_attention_t(const AttnLaunch& a, cudaStream_t stream) {
+  using Cfg = AttnCfg<DH>;
+  static bool attr_set = false;
+  auto kern = attention_kernel<DH>;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES);
+    if (e != cudaSuccess) {
+      set_last_cuda_error((int)e);
+      return XEMA_ECUDA;
+    }
+    attr_set = true;
+  }
+  AttnParams p;
+  p.o = (__nv_bfloat16*)a.o;
+  p.lse = a.lse;
+  p.batch = a.batch;
+  p.rows = a.rows;
+  p.keys = a.keys;
+  p.heads = a.heads;
+  p.scale = 1.0f / sqrtf((float)DH);
+  p.scale_log2 = p.scale * 1.4426950408889634f;
+  p.status = a.status;
+  dim3 grid((a.rows + ATT_BM - 1) / ATT_BM, a.heads, a.batch);
+  kern<<<grid, ATT_THREADS, Cfg::SMEM_BYTES, stream>>>(a.map_q, a.map_k, a.map_v, p);
+  return check_launch();
+}
+
+int launch_attention(const AttnLaunch& a, cudaStream_t stream) {
+  if (a.rows == 0 || a.batch == 0) return XEMA_OK;
+  if (a.head_dim == 64) return launch_attention_t<64>(a, stream);
+  if (a.head_dim == 128) return launch_attention_t<128>(a, stream);
+  return XEMA_EINVAL;
+}
+
+int attn_prepare(AttnLaunch* a, const void* q, long long ldq, long long q_batch_rows, const void* k, const void* v,
+                 long long ldkv, long long kv_batch_rows) {
+  if (a->batch < 1 || a->rows < 0 || a->keys < 1 || a->heads < 1) return XEMA_EINVAL;
+  if (a->head_dim != 64 && a->head_dim != 128) return XEMA_EINVAL;
+  if (a->heads > 65535 || a->batch > 65535) return XEMA_EINVAL;
+  if (!q || !k || !v || !a->o) return XEMA_EINVAL;
+  if ((ldq & 7) || (ldkv & 7)) return XEMA_EALIGN;
+  auto mis = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) != 0; };
+  if (mis(q) || mis(k) || mis(v) || mis(a->o)) return XEMA_EALIGN;
+  const long long width = (long long)a->heads * a->head_dim;
+  int rc = encode_tmap_bf16(&a->map_q, q, width, a->rows > 0 ? a->rows : 1, a->batch, ldq, q_batch_rows, ATT_BM);
+  if (rc) return rc;
+  rc = encode_tmap_bf16(&a->map_k, k, width, a->keys, a->batch, ldkv, kv_batch_rows, ATT_BN);
+  if (rc) return rc;
+  return encode_tmap_bf16(&a->map_v, v, width, a->keys, a->batch, ldkv, kv_batch_rows, ATT_BN);
+}
+
+}  // namespace xema

@@ -1,0 +1,361 @@
+// bf16 x bf16 -> fp32 GEMM on the 5th-generation tensor cores (tcgen05) with the four fused
+// epilogues of the DiT block.
+//
+//   acc[b, i, n] = sum_k A[b, i, k] * W[n, k]          (both operands K-major)
+//
+// Structure of one CTA (persistent, one per SM, 192 threads):
+//   warp 0    TMA producer: 128 x 64 tiles of A and BN x 64 tiles of W into a ring of
+//             shared-memory stages (128-byte swizzle), completion on mbarriers
+//   warp 1    owns TMEM; one thread issues tcgen05.mma (M = 128, N = BN, K = 16) into one of
+//             two fp32 accumulators in TMEM and commits stage releases / accumulator-ready
+//   warps 2-5 epilogue: tcgen05.ld the finished accumulator (thread = output row), apply the
+//             epilogue in fp32 and store; runs while the next tile's main loop fills the
+//             other accumulator
+// A row's result depends only on (row, N, K): the K loop always runs in the same order and the
+// tile shape is chosen from N alone, so outputs are bit-identical however rows are chunked.
+#include "kernels.h"
+#include "sm100.cuh"
+
+namespace xema {
+using namespace sm100;
+
+constexpr int BM = 128;
+constexpr int BK = 64;
+constexpr int GEMM_THREADS = 192;
+constexpr int GROUP_M = 8;
+constexpr int A_TILE_BYTES = BM * BK * 2;
+
+template <int BN>
+struct GemmCfg {
+  static constexpr int B_TILE_BYTES = BN * BK * 2;
+  static constexpr int STAGE_BYTES = A_TILE_BYTES + B_TILE_BYTES;
+  static constexpr int STAGES = (BN == 256) ? 4 : 6;
+  static constexpr int TMEM_COLS = 2 * BN;
+  static constexpr int BAR_BYTES = 256;
+  static constexpr int SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + BAR_BYTES;
+};
+
+struct GemmParams {
+  const __nv_bfloat16* bias;
+  void* out;
+  long long ldo, out_batch_rows;
+  const void* resid;
+  long long ldr, resid_batch_rows;
+  const float* gate;
+  long long gate_stride;
+  int batch, rows, N, K;
+  unsigned int* status;
+};
+
+__device__ __forceinline__ float gelu_tanh_f(float z) {
+  const float u = 0.7978845608028654f * fmaf(0.044715f * z * z, z, z);
+  return 0.5f * z * (1.f + tanh_approx(u));
+}
+
+template <int EPI>
+__device__ __forceinline__ void epilogue_chunk(const GemmParams& p, int b, int row, int n0, const uint32_t (&r)[32]) {
+  // bias and gate are the same for every row of the tile: broadcast loads
+  float v[32];
+  const uint4* bp = reinterpret_cast<const uint4*>(p.bias + n0);
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const uint4 bb = __ldg(bp + q);
+    v[8 * q + 0] = __uint_as_float(r[8 * q + 0]) + bf16_lo(bb.x);
+    v[8 * q + 1] = __uint_as_float(r[8 * q + 1]) + bf16_hi(bb.x);
+    v[8 * q + 2] = __uint_as_float(r[8 * q + 2]) + bf16_lo(bb.y);
+    v[8 * q + 3] = __uint_as_float(r[8 * q + 3]) + bf16_hi(bb.y);
+    v[8 * q + 4] = __uint_as_float(r[8 * q + 4]) + bf16_lo(bb.z);
+    v[8 * q + 5] = __uint_as_float(r[8 * q + 5]) + bf16_hi(bb.z);
+    v[8 * q + 6] = __uint_as_float(r[8 * q + 6]) + bf16_lo(bb.w);
+    v[8 * q + 7] = __uint_as_float(r[8 * q + 7]) + bf16_hi(bb.w);
+  }
+  if (row >= p.rows) return;
+  const size_t orow = ((size_t)b * p.out_batch_rows + row) * p.ldo + n0;
+  if constexpr (EPI == XEMA_EPI_BIAS || EPI == XEMA_EPI_BIAS_GELU) {
+    if constexpr (EPI == XEMA_EPI_BIAS_GELU) {
+#pragma unroll
+      for (int t = 0; t < 32; ++t) v[t] = gelu_tanh_f(v[t]);
+    }
+    uint4* op = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.out) + orow);
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+      op[q] = make_uint4(pack_bf16x2(v[8 * q], v[8 * q + 1]), pack_bf16x2(v[8 * q + 2], v[8 * q + 3]),
+                         pack_bf16x2(v[8 * q + 4], v[8 * q + 5]), pack_bf16x2(v[8 * q + 6], v[8 * q + 7]));
+  } else {
+    const float4* gp = reinterpret_cast<const float4*>(p.gate + (size_t)b * p.gate_stride + n0);
+    const size_t rrow = ((size_t)b * p.resid_batch_rows + row) * p.ldr + n0;
+    if constexpr (EPI == XEMA_EPI_GATE_RES_F32) {
+      // out fp32 = resid(bf16) + gate * v
+      const uint4* rp = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(p.resid) + rrow);
+      float4* op = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + orow);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const uint4 x = __ldg(rp + q);
+        const float4 g0 = __ldg(gp + 2 * q), g1 = __ldg(gp + 2 * q + 1);
+        op[2 * q] = make_float4(fmaf(g0.x, v[8 * q + 0], bf16_lo(x.x)), fmaf(g0.y, v[8 * q + 1], bf16_hi(x.x)),
+                                fmaf(g0.z, v[8 * q + 2], bf16_lo(x.y)), fmaf(g0.w, v[8 * q + 3], bf16_hi(x.y)));
+        op[2 * q + 1] = make_float4(fmaf(g1.x, v[8 * q + 4], bf16_lo(x.z)), fmaf(g1.y, v[8 * q + 5], bf16_hi(x.z)),
+                                    fmaf(g1.z, v[8 * q + 6], bf16_lo(x.w)), fmaf(g1.w, v[8 * q + 7], bf16_hi(x.w)));
+      }
+    } else {
+      // out bf16 = resid(fp32) + gate * v
+      const float4* rp = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(p.resid) + rrow);
+      uint4* op = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.out) + orow);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const float4 x0 = __ldg(rp + 2 * q), x1 = __ldg(rp + 2 * q + 1);
+        const float4 g0 = __ldg(gp + 2 * q), g1 = __ldg(gp + 2 * q + 1);
+        op[q] = make_uint4(
+            pack_bf16x2(fmaf(g0.x, v[8 * q + 0], x0.x), fmaf(g0.y, v[8 * q + 1], x0.y)),
+            pack_bf16x2(fmaf(g0.z, v[8 * q + 2], x0.z), fmaf(g0.w, v[8 * q + 3], x0.w)),
+            pack_bf16x2(fmaf(g1.x, v[8 * q + 4], x1.x), fmaf(g1.y, v[8 * q + 5], x1.y)),
+            pack_bf16x2(fmaf(g1.z, v[8 * q + 6], x1.z), fmaf(g1.w, v[8 * q + 7], x1.w)));
+      }
+    }
+  }
+}
+
+struct TileCoord {
+  int b, mt, nt;
+};
+__device__ __forceinline__ TileCoord tile_coord(int tile, int m_tiles, int n_tiles) {
+  const int per_batch = m_tiles * n_tiles;
+  TileCoord c;
+  c.b = tile / per_batch;
+  const int t = tile - c.b * per_batch;
+  const int group_size = GROUP_M * n_tiles;
+  const int g = t / group_size;
+  const int first_m = g * GROUP_M;
+  const int gm = min(GROUP_M, m_tiles - first_m);
+  const int in_group = t - g * group_size;
+  c.mt = first_m + in_group % gm;
+  c.nt = in_group / gm;
+  return c;
+}
+
+template <int BN, int EPI>
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+gemm_bf16_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w,
+                 const GemmParams p) {
+  using Cfg = GemmCfg<BN>;
+  constexpr int STAGES = Cfg::STAGES;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* bar_base = smem + STAGES * Cfg::STAGE_BYTES;
+  uint64_t* full = reinterpret_cast<uint64_t*>(bar_base);
+  uint64_t* empty = full + STAGES;
+  uint64_t* tmem_full = empty + STAGES;
+  uint64_t* tmem_empty = tmem_full + 2;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tmem_empty + 2);
+  volatile uint32_t* abort_flag = tmem_slot + 1;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int m_tiles = (p.rows + BM - 1) / BM;
+  const int n_tiles = p.N / BN;
+  const int k_blocks = p.K / BK;
+  const int total_tiles = p.batch * m_tiles * n_tiles;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(&full[s], 1);
+      mbar_init(&empty[s], 1);
+    }
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(&tmem_full[s], 1);
+      mbar_init(&tmem_empty[s], 4);
+    }
+    *abort_flag = 0;
+    fence_mbar_init();
+    prefetch_tmap(&map_a);
+    prefetch_tmap(&map_w);
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_slot, Cfg::TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+        const TileCoord c = tile_coord(tile, m_tiles, n_tiles);
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          if (!(ok = mbar_wait(&empty[stage], phase ^ 1, abort_flag))) break;
+          uint8_t* sa = smem + stage * Cfg::STAGE_BYTES;
+          uint8_t* sb = sa + A_TILE_BYTES;
+          mbar_expect_tx(&full[stage], Cfg::STAGE_BYTES);
+          tma_load_3d(sa, &map_a, &full[stage], kb * BK, c.mt * BM, c.b);
+          tma_load_3d(sb, &map_w, &full[stage], kb * BK, c.nt * BN, 0);
+          if (++stage == STAGES) { stage = 0; phase ^= 1; }
+        }
+      }
+      if (!ok) {
+        // gave up: let the copies already issued land before the CTA leaves
+        for (int s = 0; s < STAGES; ++s) {
+          const int st = (stage + s) % STAGES;                 // oldest outstanding first
+          const uint32_t ph = (st < stage) ? phase : (phase ^ 1);
+          volatile uint32_t dummy = 0;
+          mbar_wait(&full[st], ph, &dummy);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      constexpr uint32_t idesc = idesc_bf16_f32(BM, BN, false, false);
+      int stage = 0;
+      uint32_t phase = 0;
+      int acc = 0;
+      uint32_t acc_phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+        if (!(ok = mbar_wait(&tmem_empty[acc], acc_phase ^ 1, abort_flag))) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * BN;
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          if (!(ok = mbar_wait(&full[stage], phase, abort_flag))) break;
+          tc_fence_after();
+          const uint32_t a_addr = smem_u32(smem + stage * Cfg::STAGE_BYTES);
+          const uint32_t b_addr = a_addr + A_TILE_BYTES;
+#pragma unroll
+          for (int k = 0; k < BK / 16; ++k) {
+            const uint64_t da = smem_desc_sw128(a_addr + k * 32, 16, 1024);
+            const uint64_t db = smem_desc_sw128(b_addr + k * 32, 16, 1024);
+            mma_ss(d_tmem, da, db, idesc, (kb | k) != 0);
+          }
+          mma_commit(&empty[stage]);
+          if (++stage == STAGES) { stage = 0; phase ^= 1; }
+        }
+        if (!ok) break;
+        mma_commit(&tmem_full[acc]);
+        if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+      }
+    }
+  } else {
+    // ---------------- epilogue ----------------
+    const int quad = warp & 3;           // TMEM lanes [32*quad, 32*quad + 32) belong to this warp
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+      const TileCoord c = tile_coord(tile, m_tiles, n_tiles);
+      ok = mbar_wait(&tmem_full[acc], acc_phase, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      const int row = c.mt * BM + quad * 32 + lane;
+      const uint32_t t_addr = tmem_base + ((uint32_t)(quad * 32) << 16) + acc * BN;
+#pragma unroll 1
+      for (int ch = 0; ch < BN / 32; ++ch) {
+        uint32_t r[32];
+        tmem_ld32(t_addr + ch * 32, r);
+        tmem_ld_wait();
+        epilogue_chunk<EPI>(p, c.b, row, c.nt * BN + ch * 32, r);
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&tmem_empty[acc]);
+      if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, Cfg::TMEM_COLS);
+  }
+  if (threadIdx.x == 0 && *abort_flag && p.status) atomicExch(p.status, STATUS_TIMEOUT_MBARRIER);
+}
+
+// ---------------------------------------------------------------------------------------------
+static int g_sm_count = 0;
+static int sm_count() {
+  if (g_sm_count == 0) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return 148;
+    g_sm_count = n;
+  }
+  return g_sm_count;
+}
+
+template <int BN, int EPI>
+static int launch_gemm_t(const GemmLaunch& g, cudaStream_t stream) {
+  using Cfg = GemmCfg<BN>;
+  static bool attr_set = false;
+  auto kern = gemm_bf16_kernel<BN, EPI>;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES);
+    if (e != cudaSuccess) {
+      set_last_cuda_error((int)e);
+      return XEMA_ECUDA;
+    }
+    attr_set = true;
+  }
+  GemmParams p;
+  p.bias = (const __nv_bfloat16*)g.bias;
+  p.out = g.out;
+  p.ldo = g.ldo;
+  p.out_batch_rows = g.out_batch_rows;
+  p.resid = g.resid;
+  p.ldr = g.ldr;
+  p.resid_batch_rows = g.resid_batch_rows;
+  p.gate = g.gate;
+  p.gate_stride = g.gate_stride;
+  p.batch = g.batch;
+  p.rows = g.rows;
+  p.N = g.N;
+  p.K = g.K;
+  p.status = g.status;
+  const int m_tiles = (g.rows + BM - 1) / BM;
+  const long long tiles = (long long)g.batch * m_tiles * (g.N / BN);
+  const int grid = (int)std::min<long long>(tiles, sm_count());
+  kern<<<grid, GEMM_THREADS, Cfg::SMEM_BYTES, stream>>>(g.map_a, g.map_w, p);
+  return check_launch();
+}
+
+template <int BN>
+static int launch_gemm_bn(const GemmLaunch& g, cudaStream_t stream) {
+  switch (g.epilogue) {
+    case XEMA_EPI_BIAS: return launch_gemm_t<BN, XEMA_EPI_BIAS>(g, stream);
+    case XEMA_EPI_BIAS_GELU: return launch_gemm_t<BN, XEMA_EPI_BIAS_GELU>(g, stream);
+    case XEMA_EPI_GATE_RES_F32: return launch_gemm_t<BN, XEMA_EPI_GATE_RES_F32>(g, stream);
+    case XEMA_EPI_GATE_RES_BF16: return launch_gemm_t<BN, XEMA_EPI_GATE_RES_BF16>(g, stream);
+    default: return XEMA_EINVAL;
+  }
+}
+
+int launch_gemm(const GemmLaunch& g, cudaStream_t stream) {
+  if (g.rows == 0 || g.batch == 0) return XEMA_OK;
+  if (g.block_n == 256) return launch_gemm_bn<256>(g, stream);
+  if (g.block_n == 128) return launch_gemm_bn<128>(g, stream);
+  return XEMA_EINVAL;
+}
+
+int gemm_prepare(GemmLaunch* g, const void* a, long long lda, long long a_batch_rows, const void* w, long long ldw) {
+  if (g->batch < 1 || g->rows < 0 || g->N < 128 || (g->N % 128) || g->K < 64 || (g->K % 64)) return XEMA_EINVAL;
+  if (g->epilogue < XEMA_EPI_BIAS || g->epilogue > XEMA_EPI_GATE_RES_BF16) return XEMA_EINVAL;
+  if (!a || !w || !g->bias || !g->out) return XEMA_EINVAL;
+  if (g->epilogue >= XEMA_EPI_GATE_RES_F32 && (!g->resid || !g->gate)) return XEMA_EINVAL;
+  if ((lda & 7) || (ldw & 7) || (g->ldo & 7) || (g->epilogue >= XEMA_EPI_GATE_RES_F32 && (g->ldr & 7)))
+    return XEMA_EALIGN;
+  auto mis = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) != 0; };
+  if (mis(a) || mis(w) || mis(g->bias) || mis(g->out) || (g->resid && mis(g->resid)) || (g->gate && mis(g->gate)))
+    return XEMA_EALIGN;
+  // tile width from N alone, so the arithmetic of a row never depends on how rows are chunked
+  g->block_n = (g->N % 256 == 0) ? 256 : 128;
+  int rc = encode_tmap_bf16(&g->map_a, a, g->K, g->rows > 0 ? g->rows : 1, g->batch, lda, a_batch_rows, BM);
+  if (rc) return rc;
+  return encode_tmap_bf16(&g->map_w, w, g->K, g->N, 1, ldw, g->N, g->block_n);
+}
+
+}  // namespace xema

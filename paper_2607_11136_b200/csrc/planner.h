@@ -1,0 +1,18 @@
+// Internal C++ view of the host planner (trace, Algorithm 1 layout, chunk search).
+#pragma once
+#include <vector>
+
+#include "../../include/xema.h"
+
+namespace xema {
+
+int validate_config(const xema_config& cfg);
+int64_t seq_len(const xema_config& cfg);
+int build_trace(const xema_config& cfg, int32_t chunks, std::vector<xema_tensor>& out, uint32_t* n_ops);
+uint64_t max_live(const xema_tensor* t, size_t n);
+int plan_arena(const xema_tensor* t, size_t n, uint64_t* offsets, uint64_t* peak, uint64_t* live);
+int chunks_for_budget(const xema_config& cfg, uint64_t budget, int32_t max_chunks, int32_t* chunks,
+                      uint64_t* peak_out);
+int rope_table(const xema_config& cfg, float* out);
+
+}  // namespace xema

@@ -1,0 +1,411 @@
+// Executor and C ABI: binds a plan to arena memory, pre-encodes the TMA descriptors, and
+// replays the block's launch list on the caller's stream.  Nothing here allocates, frees or
+// synchronises device memory.
+#include <cuda_bf16.h>
+
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <unordered_map>
+#include <vector>
+
+#include "kernels.h"
+#include "planner.h"
+
+namespace xema {
+
+static thread_local int t_last_cuda_error = 0;
+void set_last_cuda_error(int code) { t_last_cuda_error = code; }
+
+int check_launch() {
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) {
+    t_last_cuda_error = (int)e;
+    return XEMA_ECUDA;
+  }
+  return XEMA_OK;
+}
+
+// cuTensorMapEncodeTiled is fetched from the driver at run time so the library has no link
+// dependency on libcuda and loads on machines without a driver.
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres);
+    if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || !p) {
+      t_last_cuda_error = (int)(e != cudaSuccess ? e : cudaErrorUnknown);
+      return nullptr;
+    }
+    fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+int encode_tmap_bf16(CUtensorMap* out, const void* base, long long cols, long long rows, long long batch,
+                     long long ld, long long batch_rows, int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return XEMA_ECUDA;
+  if (cols < 64 || rows < 1 || batch < 1 || ld < cols || box_rows < 1 || box_rows > 256) return XEMA_EINVAL;
+  if ((reinterpret_cast<uintptr_t>(base) & 15) || (ld & 7)) return XEMA_EALIGN;
+  if (batch > 1 && batch_rows < rows) return XEMA_EINVAL;
+  cuuint64_t dims[3] = {(cuuint64_t)cols, (cuuint64_t)rows, (cuuint64_t)batch};
+  long long bstride = (batch_rows > 0 ? batch_rows : rows) * ld * 2;
+  cuuint64_t strides[2] = {(cuuint64_t)(ld * 2), (cuuint64_t)bstride};
+  cuuint32_t box[3] = {64u, (cuuint32_t)box_rows, 1u};
+  cuuint32_t estr[3] = {1u, 1u, 1u};
+  CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    t_last_cuda_error = (int)r;
+    return XEMA_ECUDA;
+  }
+  return XEMA_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+enum OpKind { OP_MOD, OP_LN, OP_ROPE, OP_GEMM, OP_ATTN };
+
+struct Op {
+  OpKind kind;
+  // OP_MOD
+  const void *temb, *w_mod, *b_mod;
+  float* mod;
+  // OP_LN
+  const void* ln_in;
+  int ln_in_f32;
+  long long ln_in_batch_rows;
+  void* ln_out;
+  const float *shift, *scale;
+  // OP_ROPE
+  void* rope_x;
+  long long rope_ld, rope_batch_rows;
+  const void* rope_g;
+  int pos0;
+  // shared
+  int rows;
+  GemmLaunch gemm;
+  AttnLaunch attn;
+};
+
+}  // namespace xema
+
+using namespace xema;
+
+struct xema_plan {
+  xema_config cfg;
+  int32_t chunks;
+  std::vector<xema_tensor> tensors;
+  std::vector<uint64_t> offsets;
+  std::unordered_map<std::string, size_t> index;
+  uint64_t peak, live;
+  uint32_t n_ops;
+  bool bound;
+  const float* rope;
+  std::vector<Op> ops;
+};
+
+static int issue(const xema_plan* pl, const Op& op, cudaStream_t st) {
+  const xema_config& c = pl->cfg;
+  switch (op.kind) {
+    case OP_MOD:
+      return launch_mod(op.temb, op.w_mod, op.b_mod, op.mod, c.batch, c.temb_dim, 6 * c.hidden, st);
+    case OP_LN:
+      return launch_ln_modulate(op.ln_in, op.ln_in_f32, op.ln_in_batch_rows, op.ln_out, op.shift, op.scale,
+                                6LL * c.hidden, c.batch, op.rows, c.hidden, c.ln_eps, st);
+    case OP_ROPE:
+      return launch_rmsnorm_rope(op.rope_x, op.rope_ld, op.rope_batch_rows, op.rope_g, pl->rope, op.pos0, c.batch,
+                                 op.rows, c.heads, c.head_dim, c.rms_eps, st);
+    case OP_GEMM:
+      return launch_gemm(op.gemm, st);
+    case OP_ATTN:
+      return launch_attention(op.attn, st);
+  }
+  return XEMA_EINVAL;
+}
+
+static int run_ops(const xema_plan* pl, size_t n, void* stream) {
+  if (!pl) return XEMA_EINVAL;
+  if (!pl->bound) return XEMA_ESTATE;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  n = std::min(n, pl->ops.size());
+  for (size_t i = 0; i < n; ++i) {
+    int rc = issue(pl, pl->ops[i], st);
+    if (rc) return rc;
+  }
+  return XEMA_OK;
+}
+
+extern "C" {
+
+int xema_plan_create(const xema_config* cfg, int32_t chunks, xema_plan** out) {
+  if (!cfg || !out) return XEMA_EINVAL;
+  *out = nullptr;
+  xema_plan* pl = new (std::nothrow) xema_plan();
+  if (!pl) return XEMA_ENOSPC;
+  pl->cfg = *cfg;
+  pl->chunks = chunks;
+  pl->bound = false;
+  pl->rope = nullptr;
+  int rc = build_trace(*cfg, chunks, pl->tensors, &pl->n_ops);
+  if (!rc) {
+    pl->offsets.assign(pl->tensors.size(), 0);
+    rc = plan_arena(pl->tensors.data(), pl->tensors.size(), pl->offsets.data(), &pl->peak, &pl->live);
+  }
+  if (rc) {
+    delete pl;
+    return rc;
+  }
+  for (size_t i = 0; i < pl->tensors.size(); ++i) pl->index[pl->tensors[i].name] = i;
+  *out = pl;
+  return XEMA_OK;
+}
+
+void xema_plan_destroy(xema_plan* plan) { delete plan; }
+
+int xema_plan_info(const xema_plan* plan, uint64_t* peak_bytes, uint64_t* max_live_bytes, size_t* n_tensors,
+                   uint32_t* n_ops, int32_t* chunks) {
+  if (!plan) return XEMA_EINVAL;
+  if (peak_bytes) *peak_bytes = plan->peak;
+  if (max_live_bytes) *max_live_bytes = plan->live;
+  if (n_tensors) *n_tensors = plan->tensors.size();
+  if (n_ops) *n_ops = plan->n_ops;
+  if (chunks) *chunks = plan->chunks;
+  return XEMA_OK;
+}
+
+int xema_plan_tensor(const xema_plan* plan, const char* name, uint64_t* offset, uint64_t* bytes) {
+  if (!plan || !name) return XEMA_EINVAL;
+  auto it = plan->index.find(name);
+  if (it == plan->index.end()) return XEMA_EINVAL;
+  if (offset) *offset = plan->offsets[it->second];
+  if (bytes) *bytes = plan->tensors[it->second].bytes;
+  return XEMA_OK;
+}
+
+int xema_plan_tensor_at(const xema_plan* plan, size_t i, xema_tensor* tensor, uint64_t* offset) {
+  if (!plan || i >= plan->tensors.size()) return XEMA_EINVAL;
+  if (tensor) *tensor = plan->tensors[i];
+  if (offset) *offset = plan->offsets[i];
+  return XEMA_OK;
+}
+
+int xema_plan_bind(xema_plan* plan, void* arena_dev, uint64_t arena_bytes, const xema_block_weights* weights,
+                   const float* rope_dev, void* status_dev) {
+  if (!plan || !arena_dev || !weights || !rope_dev) return XEMA_EINVAL;
+  if (arena_bytes < plan->peak) return XEMA_ENOSPC;
+  if (reinterpret_cast<uintptr_t>(arena_dev) & 255) return XEMA_EALIGN;
+  if (reinterpret_cast<uintptr_t>(rope_dev) & 15) return XEMA_EALIGN;
+  const xema_config& c = plan->cfg;
+  if (c.hidden % 256 || c.ffn % 256 || c.temb_dim % 8 || (c.head_dim != 64 && c.head_dim != 128))
+    return XEMA_EINVAL;
+  plan->bound = false;
+  plan->ops.clear();
+  plan->rope = rope_dev;
+  uint8_t* arena = static_cast<uint8_t*>(arena_dev);
+  unsigned int* status = static_cast<unsigned int*>(status_dev);
+
+  auto at = [&](const char* stem, int block, int chunk) -> uint8_t* {
+    char name[32];
+    if (block < 0)
+      std::snprintf(name, sizeof(name), "%s", stem);
+    else if (chunk < 0)
+      std::snprintf(name, sizeof(name), "%s%d", stem, block);
+    else
+      std::snprintf(name, sizeof(name), "%s%d_%d", stem, block, chunk);
+    auto it = plan->index.find(name);
+    if (it == plan->index.end()) return nullptr;
+    const size_t i = it->second;
+    if (plan->offsets[i] + plan->tensors[i].bytes > arena_bytes) return nullptr;
+    return arena + plan->offsets[i];
+  };
+
+  const long long S = seq_len(c), D = c.hidden, F = c.ffn;
+  const int C = plan->chunks;
+  for (int l = 0; l < c.n_blocks; ++l) {
+    const xema_block_weights& w = weights[l];
+    const void* wp[12] = {w.w_mod, w.b_mod, w.w_qkv, w.b_qkv, w.g_q, w.g_k, w.w_o, w.b_o, w.w_1, w.b_1, w.w_2, w.b_2};
+    for (const void* p : wp) {
+      if (!p) return XEMA_EINVAL;
+      if (reinterpret_cast<uintptr_t>(p) & 15) return XEMA_EALIGN;
+    }
+    const __nv_bfloat16* w_qkv = static_cast<const __nv_bfloat16*>(w.w_qkv);
+    const __nv_bfloat16* b_qkv = static_cast<const __nv_bfloat16*>(w.b_qkv);
+    uint8_t* hid = at("hid", l, -1);
+    uint8_t* hid_next = at("hid", l + 1, -1);
+    float* mod = reinterpret_cast<float*>(at("mod", l, -1));
+    uint8_t* kv = at("kv", l, -1);
+    uint8_t* res = at("res", l, -1);
+    uint8_t* temb = at("temb", -1, -1);
+    if (!hid || !hid_next || !mod || !kv || !res || !temb) return XEMA_EINVAL;
+
+    Op op{};
+    op.kind = OP_MOD;
+    op.temb = temb; op.w_mod = w.w_mod; op.b_mod = w.b_mod; op.mod = mod;
+    plan->ops.push_back(op);
+
+    auto ln_op = [&](const void* in, int f32, void* out, int rows, int which) {
+      Op o{};
+      o.kind = OP_LN;
+      o.ln_in = in; o.ln_in_f32 = f32; o.ln_in_batch_rows = S; o.ln_out = out;
+      o.shift = mod + (which == 1 ? 0 : 3 * D);
+      o.scale = mod + (which == 1 ? D : 4 * D);
+      o.rows = rows;
+      plan->ops.push_back(o);
+    };
+    auto gemm_op = [&](const void* a, long long lda, long long a_batch_rows, const void* wt, long long ldw,
+                       const void* bias, void* out, long long ldo, long long out_batch_rows, const void* resid,
+                       long long ldr, long long resid_batch_rows, const float* gate, int rows, int N, int K,
+                       int epi) -> int {
+      Op o{};
+      o.kind = OP_GEMM;
+      GemmLaunch& g = o.gemm;
+      g.bias = bias; g.out = out; g.ldo = ldo; g.out_batch_rows = out_batch_rows;
+      g.resid = resid; g.ldr = ldr; g.resid_batch_rows = resid_batch_rows;
+      g.gate = gate; g.gate_stride = 6 * D;
+      g.batch = c.batch; g.rows = rows; g.N = N; g.K = K; g.epilogue = epi; g.status = status;
+      int rc = gemm_prepare(&g, a, lda, a_batch_rows, wt, ldw);
+      if (rc) return rc;
+      plan->ops.push_back(o);
+      return XEMA_OK;
+    };
+
+    // phase A: keys and values of every chunk
+    for (int ci = 0; ci < C; ++ci) {
+      const long long r0 = (long long)ci * S / C, r1 = (long long)(ci + 1) * S / C;
+      const int n = (int)(r1 - r0);
+      uint8_t* h1a = at("h1a", l, ci);
+      if (!h1a) return XEMA_EINVAL;
+      ln_op(hid + r0 * D * 2, 0, h1a, n, 1);
+      int rc = gemm_op(h1a, D, n, w_qkv + D * D, D, b_qkv + D, kv + r0 * 2 * D * 2, 2 * D, S, nullptr, 0, 0, nullptr,
+                       n, (int)(2 * D), (int)D, XEMA_EPI_BIAS);
+      if (rc) return rc;
+      Op o{};
+      o.kind = OP_ROPE;
+      o.rope_x = kv + r0 * 2 * D * 2; o.rope_ld = 2 * D; o.rope_batch_rows = S; o.rope_g = w.g_k;
+      o.pos0 = (int)r0; o.rows = n;
+      plan->ops.push_back(o);
+    }
+    // phase B: queries, attention and the gated output projection of every chunk
+    for (int ci = 0; ci < C; ++ci) {
+      const long long r0 = (long long)ci * S / C, r1 = (long long)(ci + 1) * S / C;
+      const int n = (int)(r1 - r0);
+      uint8_t* h1b = at("h1b", l, ci);
+      uint8_t* q = at("q", l, ci);
+      uint8_t* o_t = at("o", l, ci);
+      float* lse = reinterpret_cast<float*>(at("lse", l, ci));
+      if (!h1b || !q || !o_t || !lse) return XEMA_EINVAL;
+      ln_op(hid + r0 * D * 2, 0, h1b, n, 1);
+      int rc = gemm_op(h1b, D, n, w_qkv, D, b_qkv, q, D, n, nullptr, 0, 0, nullptr, n, (int)D, (int)D, XEMA_EPI_BIAS);
+      if (rc) return rc;
+      Op o{};
+      o.kind = OP_ROPE;
+      o.rope_x = q; o.rope_ld = D; o.rope_batch_rows = n; o.rope_g = w.g_q; o.pos0 = (int)r0; o.rows = n;
+      plan->ops.push_back(o);
+      Op a{};
+      a.kind = OP_ATTN;
+      a.attn.o = o_t; a.attn.lse = lse; a.attn.batch = c.batch; a.attn.rows = n; a.attn.keys = (int)S;
+      a.attn.heads = c.heads; a.attn.head_dim = c.head_dim; a.attn.status = status;
+      rc = attn_prepare(&a.attn, q, D, n, kv, kv + D * 2, 2 * D, S);
+      if (rc) return rc;
+      plan->ops.push_back(a);
+      rc = gemm_op(o_t, D, n, w.w_o, D, w.b_o, res + r0 * D * 4, D, S, hid + r0 * D * 2, D, S, mod + 2 * D, n, (int)D,
+                   (int)D, XEMA_EPI_GATE_RES_F32);
+      if (rc) return rc;
+    }
+    // phase C: feed-forward of every chunk
+    for (int ci = 0; ci < C; ++ci) {
+      const long long r0 = (long long)ci * S / C, r1 = (long long)(ci + 1) * S / C;
+      const int n = (int)(r1 - r0);
+      uint8_t* h2 = at("h2", l, ci);
+      uint8_t* g = at("g", l, ci);
+      if (!h2 || !g) return XEMA_EINVAL;
+      ln_op(res + r0 * D * 4, 1, h2, n, 2);
+      int rc = gemm_op(h2, D, n, w.w_1, D, w.b_1, g, F, n, nullptr, 0, 0, nullptr, n, (int)F, (int)D,
+                       XEMA_EPI_BIAS_GELU);
+      if (rc) return rc;
+      rc = gemm_op(g, F, n, w.w_2, F, w.b_2, hid_next + r0 * D * 2, D, S, res + r0 * D * 4, D, S, mod + 5 * D, n,
+                   (int)D, (int)F, XEMA_EPI_GATE_RES_BF16);
+      if (rc) return rc;
+    }
+  }
+  if (plan->ops.size() != plan->n_ops) return XEMA_EINVAL;
+  plan->bound = true;
+  return XEMA_OK;
+}
+
+int xema_block_forward(const xema_plan* plan, void* stream) {
+  if (!plan) return XEMA_EINVAL;
+  if (plan->cfg.n_blocks != 1) return XEMA_ESTATE;
+  return run_ops(plan, plan->ops.size(), stream);
+}
+
+int xema_step_forward(const xema_plan* plan, void* stream) {
+  if (!plan) return XEMA_EINVAL;
+  return run_ops(plan, plan->ops.size(), stream);
+}
+
+int xema_forward_prefix(const xema_plan* plan, uint32_t n_logical_ops, void* stream) {
+  return run_ops(plan, n_logical_ops, stream);
+}
+
+int xema_plan_launch_count(const xema_plan* plan) {
+  return (plan && plan->bound) ? (int)plan->ops.size() : 0;
+}
+
+int xema_op_mod(const void* temb, const void* w_mod, const void* b_mod, float* mod, int32_t batch, int32_t temb_dim,
+                int32_t n_out, void* stream) {
+  if (!temb || !w_mod || !b_mod || !mod) return XEMA_EINVAL;
+  return launch_mod(temb, w_mod, b_mod, mod, batch, temb_dim, n_out, reinterpret_cast<cudaStream_t>(stream));
+}
+
+int xema_op_ln_modulate(const void* in, int32_t in_is_f32, int64_t in_batch_rows, void* out, const float* shift,
+                        const float* scale, int64_t mod_stride, int32_t batch, int32_t rows, int32_t D, float eps,
+                        void* stream) {
+  if (!in || !out || !shift || !scale) return XEMA_EINVAL;
+  return launch_ln_modulate(in, in_is_f32, in_batch_rows, out, shift, scale, mod_stride, batch, rows, D, eps,
+                            reinterpret_cast<cudaStream_t>(stream));
+}
+
+int xema_op_rmsnorm_rope(void* x, int64_t ld, int64_t batch_rows, const void* g, const float* rope, int32_t pos0,
+                         int32_t batch, int32_t rows, int32_t heads, int32_t head_dim, float eps, void* stream) {
+  if (!x || !g || !rope) return XEMA_EINVAL;
+  return launch_rmsnorm_rope(x, ld, batch_rows, g, rope, pos0, batch, rows, heads, head_dim, eps,
+                             reinterpret_cast<cudaStream_t>(stream));
+}
+
+int xema_op_gemm(const xema_gemm_args* a, void* status_dev, void* stream) {
+  if (!a) return XEMA_EINVAL;
+  GemmLaunch g{};
+  g.bias = a->bias; g.out = a->out; g.ldo = a->ldo; g.out_batch_rows = a->out_batch_rows;
+  g.resid = a->resid; g.ldr = a->ldr; g.resid_batch_rows = a->resid_batch_rows;
+  g.gate = a->gate; g.gate_stride = a->gate_stride;
+  g.batch = a->batch; g.rows = a->rows; g.N = a->N; g.K = a->K; g.epilogue = a->epilogue;
+  g.status = static_cast<unsigned int*>(status_dev);
+  int rc = gemm_prepare(&g, a->a, a->lda, a->a_batch_rows, a->w, a->ldw);
+  if (rc) return rc;
+  return launch_gemm(g, reinterpret_cast<cudaStream_t>(stream));
+}
+
+int xema_op_attention(const void* q, int64_t ldq, int64_t q_batch_rows, const void* k, const void* v, int64_t ldkv,
+                      int64_t kv_batch_rows, void* o, float* lse, int32_t batch, int32_t rows, int32_t keys,
+                      int32_t heads, int32_t head_dim, void* status_dev, void* stream) {
+  AttnLaunch a{};
+  a.o = o; a.lse = lse; a.batch = batch; a.rows = rows; a.keys = keys; a.heads = heads; a.head_dim = head_dim;
+  a.status = static_cast<unsigned int*>(status_dev);
+  int rc = attn_prepare(&a, q, ldq, q_batch_rows, k, v, ldkv, kv_batch_rows);
+  if (rc) return rc;
+  return launch_attention(a, reinterpret_cast<cudaStream_t>(stream));
+}
+
+int xema_last_cuda_error(void) { return t_last_cuda_error; }
+
+}  // extern "C"

@@ -1,0 +1,95 @@
+"""Bit-exact parity of the library's host planner with the oracle (CPU only)."""
+import math
+
+import numpy as np
+import pytest
+
+from oracle import arena as o_arena
+from oracle import block as o_block
+from oracle import trace as o_trace
+from paper_2607_11136_b200 import binding as xb
+from xema_inputs import template
+
+CASES = [("tiny", 1), ("cogvideox", 1), ("flux", 1), ("flux", 4), ("longvideo", 1), ("longvideo", 2)]
+
+
+@pytest.mark.parametrize("name,batch", CASES)
+def test_trace_offsets_peak_bit_exact(name, batch):
+    t = template(name, batch=batch)
+    cfg = xb.make_config(t)
+    for C in list(range(1, 17)) + [31, 64]:
+        want, want_ops = o_trace.trace(t, C)
+        got, got_ops = xb.xema_trace(cfg, C)
+        assert got_ops == want_ops
+        assert got == want, (name, C)
+        offs, peak, live = xb.xema_plan_arena(got)
+        w_offs, w_peak = o_arena.plan_arena(want)
+        assert offs == w_offs and peak == w_peak
+        assert live == o_arena.max_live_bytes(want, want_ops)
+
+
+@pytest.mark.parametrize("C", [1, 2, 3, 4, 8])
+def test_step_trace_bit_exact(C):
+    t = template("step")
+    want, want_ops = o_trace.trace(t, C)
+    got, got_ops = xb.xema_trace(xb.make_config(t), C)
+    assert (got, got_ops) == (want, want_ops)
+    offs, peak, _ = xb.xema_plan_arena(got)
+    w_offs, w_peak = o_arena.plan_arena(want)
+    assert offs == w_offs and peak == w_peak
+
+
+def test_plan_object_agrees_with_free_functions():
+    t = template("cogvideox")
+    cfg = xb.make_config(t)
+    p = xb.Plan(cfg, 4)
+    ts, n_ops = xb.xema_trace(cfg, 4)
+    offs, peak, live = xb.xema_plan_arena(ts)
+    assert (p.peak_bytes, p.max_live_bytes, p.n_ops, p.n_tensors, p.chunks) == (peak, live, n_ops, len(ts), 4)
+    for d, off in zip(p.tensors(), offs):
+        assert d["offset"] == off
+        assert p.tensor(d["name"]) == (off, d["bytes"])
+    p.close()
+
+
+def test_plan_arena_on_random_traces():
+    rng = np.random.default_rng(5)
+    for _ in range(200):
+        n = int(rng.integers(1, 40))
+        ts = []
+        for _ in range(n):
+            b = int(rng.integers(0, 30))
+            ts.append({"bytes": 256 * int(rng.integers(1, 50)), "birth": b, "death": b + int(rng.integers(1, 12))})
+        offs, peak, live = xb.xema_plan_arena(ts)
+        w_offs, w_peak = o_arena.plan_arena(ts)
+        assert offs == w_offs and peak == w_peak and live == o_arena.max_live_bytes(ts)
+        assert o_arena.overlapping_pairs(ts, offs) == []
+
+
+def test_chunks_for_budget_bit_exact():
+    GiB = 1 << 30
+    sweeps = [
+        ("cogvideox", 1, [764583936, 764583935, 657074688, 657074687, 601613568, 573883136, 560 << 20, 1 << 40]),
+        ("flux", 1, [24 * GiB]), ("flux", 4, [24 * GiB, 700 << 20]),
+        ("longvideo", 1, [8 * GiB, 16 * GiB, 32 * GiB, 4 * GiB, int(3.5 * GiB), int(3.25 * GiB)]),
+        ("longvideo", 2, [8 * GiB, 16 * GiB]), ("longvideo", 4, [8 * GiB, 16 * GiB, 32 * GiB]),
+        ("step", 1, [768 << 20, 640 << 20, 576 << 20]),
+        ("tiny", 1, [2076672, 1786368, 1561856, 1500000]),
+    ]
+    for name, batch, budgets in sweeps:
+        t = template(name, batch=batch)
+        cfg = xb.make_config(t)
+        for budget in budgets:
+            assert xb.xema_chunks_for_budget(cfg, budget, 16) == o_arena.chunks_for_budget(t, budget, 16), (name, budget)
+
+
+def test_rope_table_against_oracle_angles():
+    for name in ("tiny", "flux"):
+        t = template(name)
+        tab = xb.xema_rope_table(xb.make_config(t))
+        ang = o_block.rope_angles(t)
+        assert tab.shape == (t.seq, t.head_dim // 2, 2)
+        assert np.array_equal(tab[..., 0], np.cos(ang).astype(np.float32))
+        assert np.array_equal(tab[..., 1], np.sin(ang).astype(np.float32))
+    # text tokens are left unrotated
+    assert np.all(tab[:t.s_text, :, 0] == 1.0) and np.all(tab[:t.s_text, :, 1] == 0.0)
