@@ -1,0 +1,351 @@
+#!/usr/bin/env python
+"""Benchmark of the chunked, arena-placed DiT block on B200.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cogvideox] [--budget-mib M]
+  python bench.py --impl reference ...        # times the CPU oracle instead
+
+One step = one pass of the whole hot path (modulation, LayerNorm+modulate, QKV GEMMs, RMSNorm +
+RoPE, attention, gated projection, FFN) over one batch of seeded synthetic input, sequence-
+chunked with the smallest chunk count whose arena peak fits the byte budget.  Prints ONE JSON
+line (see the keys below).  Under torchrun every rank runs the same workload on its own GPU
+(independent replicas, no data-path collective); the value is the sum over ranks divided by the
+slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from xema_inputs import bits_to_f64, make_activations, make_block_weights, sample_rows, template  # noqa: E402
+
+METRIC = "DiT block TFLOP/s (bf16 in, fp32 accumulate) at a memory budget; block latency in ms_per_step"
+UNIT = "TFLOP/s"
+CPU_SAMPLE_ROWS = 1024
+
+
+def block_flops(t) -> float:
+    """Algorithmic flops of one block: the five GEMMs plus attention (4*S^2*D per batch element)."""
+    S, D, F, B = t.seq, t.hidden, t.ffn, t.batch
+    return B * (2.0 * S * D * (3 * D + D + 2 * F) + 4.0 * S * S * D) * t.n_blocks
+
+
+def sample_flops(t, n_rows) -> float:
+    """Flops the row-sampled oracle performs: k and v for every token, everything else for the
+    sampled rows only."""
+    S, D, F, B = t.seq, t.hidden, t.ffn, t.batch
+    return B * (2.0 * S * D * 2 * D + n_rows * (2.0 * D * (2 * D + 2 * F) + 4.0 * S * D))
+
+
+def load_peaks():
+    """Measured roofline denominators written by the driver; else the pool's fallback numbers."""
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_burst": float(p["bf16_tflops"]),
+                "bf16_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), "source": "measured"}
+    except Exception:
+        return {"hbm_gbs": 6650.0, "bf16_burst": 1590.0, "bf16_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons, power = [], [], set(), []
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for r in self.rows:
+            if len(r) < 7:
+                continue
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1])); power.append(float(r[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def time_oracle_sample(t, n_rows=CPU_SAMPLE_ROWS):
+    """Times the float64 oracle, as it stands, on a bounded sample of the workload: keys and
+    values of every token, then the complete block for `n_rows` seeded token rows."""
+    from oracle import block as ob
+    w = {k: bits_to_f64(v) for k, v in make_block_weights(t, 0).items()}
+    x, temb = make_activations(t)
+    x, temb = bits_to_f64(x), bits_to_f64(temb)
+    rows = sample_rows(t, n_random=n_rows)
+    t0 = time.perf_counter()
+    ob.block_forward(t, w, x, temb, rows=rows)
+    dt = time.perf_counter() - t0
+    return dt, len(rows)
+
+
+def run_reference(args):
+    """`--impl reference`: the CPU oracle on the host cores, on the same config and metric."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    t = template(args.workload)
+    cores = len(os.sched_getaffinity(0))
+    times, n_rows = [], 0
+    for i in range(args.warmup + args.steps):
+        dt, n_rows = time_oracle_sample(t, args.cpu_rows)
+        if i >= args.warmup:
+            times.append(dt)
+    mean = float(np.mean(times))
+    value = sample_flops(t, n_rows) / mean / 1e12
+    sample = ("k, v for all %d tokens plus the complete block for %d seeded token rows of one block "
+              "(%.3g of %.3g flop)" % (t.seq, n_rows, sample_flops(t, n_rows), block_flops(t)))
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": mean * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.workload, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="xema", choices=["xema", "reference"])
+    ap.add_argument("--workload", default="cogvideox", choices=["tiny", "cogvideox", "flux", "longvideo", "step"])
+    ap.add_argument("--budget-mib", type=float, default=640.0,
+                    help="activation byte budget; the smallest chunk count whose arena peak fits is used")
+    ap.add_argument("--chunks", type=int, default=0, help="force a chunk count instead of a budget")
+    ap.add_argument("--cpu-rows", type=int, default=CPU_SAMPLE_ROWS)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", action="store_true", help="also time chunk counts 1, 2, 4, 8 (outside the timed region)")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    from paper_2607_11136_b200 import binding as xb
+    from paper_2607_11136_b200.session import BlockSession
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    dev = torch.device("cuda", local)
+    torch.cuda.set_device(dev)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    t = template(args.workload)
+    cfg = xb.make_config(t)
+    budget = None if args.chunks else int(args.budget_mib * (1 << 20))
+    weights = [make_block_weights(t, l) for l in range(t.n_blocks)]
+    x_bits, temb_bits = make_activations(t)
+    sess = BlockSession(t, weights, chunks=args.chunks or None, budget_bytes=budget, device=dev)
+    n_launch = sess.plan.launch_count()
+    ops = [sess.plan.op(i) for i in range(n_launch)]
+    flops = block_flops(t)
+    stream = torch.cuda.current_stream(dev)
+    sess.set_inputs(x_bits, temb_bits)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    # ---- device-resident timing: K steps, per-op events on the launching stream ---------------
+    for _ in range(args.warmup):
+        sess.forward(stream)
+    barrier()
+    free_before, _ = torch.cuda.mem_get_info(dev)
+    sampler = ClockSampler(local)
+    sampler.start()
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(n_launch + 1)] for _ in range(args.steps)]
+    barrier()
+    for k in range(args.steps):
+        for i in range(n_launch):
+            ev[k][i].record(stream)
+            sess.plan.forward_range(i, i + 1, stream.cuda_stream)
+        ev[k][n_launch].record(stream)
+    barrier()
+    clocks = sampler.stop()
+    free_after, _ = torch.cuda.mem_get_info(dev)
+    sess.check_status()
+    total_ms = ev[0][0].elapsed_time(ev[-1][n_launch])
+    if dist is not None:
+        tt = torch.tensor([total_ms], device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        total_ms = float(tt.item())
+    ms_per_step = total_ms / args.steps
+    value = world * flops / (ms_per_step * 1e-3) / 1e12
+
+    per_op = {}
+    for i, op in enumerate(ops):
+        d = per_op.setdefault(op["name"], {"ms": 0.0, "flops": 0.0, "bytes": 0.0, "launches": 0})
+        d["ms"] += sum(ev[k][i].elapsed_time(ev[k][i + 1]) for k in range(args.steps)) / args.steps
+        d["flops"] += op["flops"]; d["bytes"] += op["bytes"]; d["launches"] += 1
+
+    # ---- end to end through the public API: pinned host -> arena, forward, output -> host ------
+    x_host = torch.from_numpy(x_bits.view(np.int16)).pin_memory()
+    temb_host = torch.from_numpy(temb_bits.view(np.int16)).pin_memory()
+    out_host = torch.empty_like(x_host).pin_memory()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def e2e_step():
+        sess.set_inputs(x_host, temb_host, non_blocking=True)
+        sess.forward(stream)
+        out_host.copy_(sess.hid_out(), non_blocking=True)
+
+    for _ in range(3):
+        e2e_step()
+    barrier()
+    e0.record(stream)
+    for _ in range(args.steps):
+        e2e_step()
+    e1.record(stream)
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+    if dist is not None:
+        tt = torch.tensor([e2e_ms], device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        e2e_ms = float(tt.item())
+    e2e_ms /= args.steps
+    h2d = int(x_host.numel() * 2 + temb_host.numel() * 2)
+    d2h = int(out_host.numel() * 2)
+
+    sweep = None
+    if args.sweep and rank == 0:
+        sweep = {}
+        dev_w = sess.weights
+        for C in (1, 2, 4, 8):
+            s2 = BlockSession(t, dev_w, chunks=C, device=dev)
+            s2.set_inputs(x_bits, temb_bits)
+            for _ in range(3):
+                s2.forward(stream)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize(dev)
+            a.record(stream)
+            for _ in range(10):
+                s2.forward(stream)
+            b.record(stream)
+            torch.cuda.synchronize(dev)
+            ms = a.elapsed_time(b) / 10
+            sweep[str(C)] = {"ms": ms, "tflops": flops / ms / 1e9, "arena_bytes": s2.plan.peak_bytes}
+            del s2
+            torch.cuda.empty_cache()
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel ---------------------------------------------------------
+    peaks = load_peaks()
+    dom = max(per_op, key=lambda n: per_op[n]["ms"])
+    d = per_op[dom]
+    per_launch_s = d["ms"] * 1e-3 / d["launches"]
+    tensor_bound = dom in ("KV", "Q", "ATTN", "PROJ", "FFN1", "FFN2")
+    if tensor_bound:
+        achieved = d["flops"] / d["launches"] / per_launch_s / 1e12
+        peak, unit, bound = peaks["bf16_sustained"], "TFLOP/s", "tensor"
+    else:
+        achieved = d["bytes"] / d["launches"] / per_launch_s / 1e9
+        peak, unit, bound = peaks["hbm_gbs"], "GB/s", "hbm"
+    roofline = {"kernel": dom, "bound": bound, "achieved": achieved, "peak": peak, "unit": unit,
+                "frac": achieved / peak, "traffic": None, "peak_source": peaks["source"] + " (sustained)",
+                "peak_burst": peaks["bf16_burst"] if tensor_bound else None,
+                "ms_per_launch": per_launch_s * 1e3, "launches_per_step": d["launches"]}
+    breakdown = {n: {"ms": round(v["ms"], 4), "share": round(v["ms"] / ms_per_step, 4),
+                     "tflops": round(v["flops"] / (v["ms"] * 1e-3) / 1e12, 1) if v["ms"] > 0 else None,
+                     "gbs": round(v["bytes"] / (v["ms"] * 1e-3) / 1e9, 1) if v["ms"] > 0 else None}
+                 for n, v in per_op.items()}
+    tensor_ms = sum(v["ms"] for n, v in per_op.items() if n in ("KV", "Q", "ATTN", "PROJ", "FFN1", "FFN2"))
+    tensor_fl = sum(v["flops"] for n, v in per_op.items() if n in ("KV", "Q", "ATTN", "PROJ", "FFN1", "FFN2"))
+
+    cpu = None
+    if not args.no_cpu_baseline:
+        dt, n_rows = time_oracle_sample(t.with_(n_blocks=1), args.cpu_rows)
+        cpu = {"value": sample_flops(t, n_rows) / dt / 1e12, "unit": UNIT, "cores": len(os.sched_getaffinity(0)),
+               "kind": "oracle", "seconds": dt,
+               "sample": "k, v for all %d tokens plus the complete block for %d seeded token rows of one block"
+                         % (t.seq, n_rows)}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": args.workload, "batch": t.batch, "tokens": t.seq, "hidden": t.hidden,
+                   "heads": t.heads, "head_dim": t.head_dim, "ffn": t.ffn, "n_blocks": t.n_blocks,
+                   "budget_bytes": budget, "chunks": sess.chunks, "arena_bytes": sess.plan.peak_bytes,
+                   "trace_max_live_bytes": sess.plan.max_live_bytes,
+                   "device_bytes_allocated_by_forward": int(free_before - free_after),
+                   "l2": "inputs larger than L2 (weights 245 MB + arena per block)",
+                   "parallelism": "replicas x%d" % world},
+        "clocks": clocks,
+        "e2e": {"value": world * flops / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": n_launch * args.steps,
+        "roofline": roofline,
+        "tensor_ops": {"tflops": tensor_fl / (tensor_ms * 1e-3) / 1e12, "ms": tensor_ms,
+                       "frac_of_sustained": tensor_fl / (tensor_ms * 1e-3) / 1e12 / peaks["bf16_sustained"],
+                       "frac_of_nominal_2250": tensor_fl / (tensor_ms * 1e-3) / 1e12 / 2250.0},
+        "per_op": breakdown,
+        "cpu_baseline": cpu,
+    }
+    if sweep:
+        line["by_chunks"] = sweep
+    print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

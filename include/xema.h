@@ -175,6 +175,16 @@ int xema_plan_launch_count(const xema_plan* plan);
 
 /* Debug aid: enqueue only the first n_logical_ops logical ops of the trace order. */
 int xema_forward_prefix(const xema_plan* plan, uint32_t n_logical_ops, void* stream);
+/* Enqueue logical ops [first_op, end_op) of the trace order (one launch each); lets a caller
+ * put its own events between ops to time them. */
+int xema_forward_range(const xema_plan* plan, uint32_t first_op, uint32_t end_op, void* stream);
+/* Describes launch i of a bound plan: name8 (host, 8 bytes) receives "MOD", "LN1A", "KV",
+ * "KROPE", "LN1B", "Q", "QROPE", "ATTN", "PROJ", "LN2", "FFN1" or "FFN2"; *flops the algorithmic
+ * floating-point operations (2 per multiply-add; attention 4*B*rows*S*D), *bytes the
+ * algorithmic HBM bytes (each operand read once, each result written once).  Any output
+ * pointer may be NULL. */
+int xema_plan_op(const xema_plan* plan, uint32_t i, char* name8, int32_t* block, int32_t* chunk,
+                 double* flops, double* bytes);
 
 /* ---- single operators (the kernels behind the forward calls, on plain device pointers) --- */
 

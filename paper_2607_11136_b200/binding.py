@@ -22,7 +22,7 @@ EXPORTS = (
     "xema_trace", "xema_plan_arena", "xema_chunks_for_budget", "xema_rope_table",
     "xema_plan_create", "xema_plan_destroy", "xema_plan_info", "xema_plan_tensor",
     "xema_plan_tensor_at", "xema_plan_bind", "xema_block_forward", "xema_step_forward",
-    "xema_plan_launch_count", "xema_forward_prefix", "xema_op_mod", "xema_op_ln_modulate",
+    "xema_plan_launch_count", "xema_forward_prefix", "xema_forward_range", "xema_plan_op", "xema_op_mod", "xema_op_ln_modulate",
     "xema_op_rmsnorm_rope", "xema_op_gemm", "xema_op_attention", "xema_strerror",
     "xema_last_cuda_error", "xema_version",
 )
@@ -92,6 +92,8 @@ def lib() -> C.CDLL:
             "xema_step_forward": [vp, vp],
             "xema_plan_launch_count": [vp],
             "xema_forward_prefix": [vp, u32, vp],
+            "xema_forward_range": [vp, u32, u32, vp],
+            "xema_plan_op": [vp, u32, C.c_char_p, P(i32), P(i32), P(C.c_double), P(C.c_double)],
             "xema_op_mod": [vp, vp, vp, vp, i32, i32, i32, vp],
             "xema_op_ln_modulate": [vp, i32, i64, vp, vp, vp, i64, i32, i32, i32, C.c_float, vp],
             "xema_op_rmsnorm_rope": [vp, i64, i64, vp, vp, i32, i32, i32, i32, i32, C.c_float, vp],
@@ -241,6 +243,17 @@ class Plan:
 
     def step_forward(self, stream: int = 0):
         _check(lib().xema_step_forward(self._h, stream), "xema_step_forward")
+
+    def forward_range(self, first_op: int, end_op: int, stream: int = 0):
+        _check(lib().xema_forward_range(self._h, first_op, end_op, stream), "xema_forward_range")
+
+    def op(self, i: int) -> dict:
+        name = C.create_string_buffer(8)
+        blk, ch, fl, by = C.c_int32(), C.c_int32(), C.c_double(), C.c_double()
+        _check(lib().xema_plan_op(self._h, i, name, C.byref(blk), C.byref(ch), C.byref(fl), C.byref(by)),
+               "xema_plan_op")
+        return {"name": name.value.decode(), "block": blk.value, "chunk": ch.value, "flops": fl.value,
+                "bytes": by.value}
 
     def forward_prefix(self, n_logical_ops: int, stream: int = 0):
         _check(lib().xema_forward_prefix(self._h, n_logical_ops, stream), "xema_forward_prefix")

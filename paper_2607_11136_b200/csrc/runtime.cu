@@ -76,6 +76,10 @@ enum OpKind { OP_MOD, OP_LN, OP_ROPE, OP_GEMM, OP_ATTN };
 
 struct Op {
   OpKind kind;
+  char name[8];       // logical op: MOD, LN1A, KV, KROPE, LN1B, Q, QROPE, ATTN, PROJ, LN2, FFN1, FFN2
+  int block, chunk;
+  double flops;       // algorithmic floating-point operations of this launch
+  double bytes;       // algorithmic HBM bytes of this launch (operands read once, results written once)
   // OP_MOD
   const void *temb, *w_mod, *b_mod;
   float* mod;
@@ -132,12 +136,12 @@ static int issue(const xema_plan* pl, const Op& op, cudaStream_t st) {
   return XEMA_EINVAL;
 }
 
-static int run_ops(const xema_plan* pl, size_t n, void* stream) {
+static int run_ops(const xema_plan* pl, size_t first, size_t n, void* stream) {
   if (!pl) return XEMA_EINVAL;
   if (!pl->bound) return XEMA_ESTATE;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   n = std::min(n, pl->ops.size());
-  for (size_t i = 0; i < n; ++i) {
+  for (size_t i = first; i < n; ++i) {
     int rc = issue(pl, pl->ops[i], st);
     if (rc) return rc;
   }
@@ -250,11 +254,18 @@ int xema_plan_bind(xema_plan* plan, void* arena_dev, uint64_t arena_bytes, const
     Op op{};
     op.kind = OP_MOD;
     op.temb = temb; op.w_mod = w.w_mod; op.b_mod = w.b_mod; op.mod = mod;
+    const double Bd = c.batch, Dd = (double)D, Fd = (double)F, Sd = (double)S;
+    auto tag = [&](Op& o, const char* nm, int chunk, double flops, double bytes) {
+      std::snprintf(o.name, sizeof(o.name), "%s", nm);
+      o.block = l; o.chunk = chunk; o.flops = flops; o.bytes = bytes;
+    };
+    tag(op, "MOD", -1, 2.0 * Bd * 6 * Dd * c.temb_dim, 2.0 * 6 * Dd * c.temb_dim + 24.0 * Bd * Dd);
     plan->ops.push_back(op);
 
-    auto ln_op = [&](const void* in, int f32, void* out, int rows, int which) {
+    auto ln_op = [&](const void* in, int f32, void* out, int rows, int which, const char* nm, int chunk) {
       Op o{};
       o.kind = OP_LN;
+      tag(o, nm, chunk, 8.0 * Bd * rows * Dd, Bd * rows * Dd * (f32 ? 6.0 : 4.0));
       o.ln_in = in; o.ln_in_f32 = f32; o.ln_in_batch_rows = S; o.ln_out = out;
       o.shift = mod + (which == 1 ? 0 : 3 * D);
       o.scale = mod + (which == 1 ? D : 4 * D);
@@ -264,9 +275,15 @@ int xema_plan_bind(xema_plan* plan, void* arena_dev, uint64_t arena_bytes, const
     auto gemm_op = [&](const void* a, long long lda, long long a_batch_rows, const void* wt, long long ldw,
                        const void* bias, void* out, long long ldo, long long out_batch_rows, const void* resid,
                        long long ldr, long long resid_batch_rows, const float* gate, int rows, int N, int K,
-                       int epi) -> int {
+                       int epi, const char* nm, int chunk) -> int {
       Op o{};
       o.kind = OP_GEMM;
+      {
+        const double out_b = (epi == XEMA_EPI_GATE_RES_F32) ? 4.0 : 2.0;
+        const double res_b = (epi == XEMA_EPI_GATE_RES_F32) ? 2.0 : (epi == XEMA_EPI_GATE_RES_BF16 ? 4.0 : 0.0);
+        tag(o, nm, chunk, 2.0 * Bd * rows * (double)N * K,
+            2.0 * Bd * rows * K + 2.0 * (double)N * K + (out_b + res_b) * Bd * rows * N);
+      }
       GemmLaunch& g = o.gemm;
       g.bias = bias; g.out = out; g.ldo = ldo; g.out_batch_rows = out_batch_rows;
       g.resid = resid; g.ldr = ldr; g.resid_batch_rows = resid_batch_rows;
@@ -284,12 +301,13 @@ int xema_plan_bind(xema_plan* plan, void* arena_dev, uint64_t arena_bytes, const
       const int n = (int)(r1 - r0);
       uint8_t* h1a = at("h1a", l, ci);
       if (!h1a) return XEMA_EINVAL;
-      ln_op(hid + r0 * D * 2, 0, h1a, n, 1);
+      ln_op(hid + r0 * D * 2, 0, h1a, n, 1, "LN1A", ci);
       int rc = gemm_op(h1a, D, n, w_qkv + D * D, D, b_qkv + D, kv + r0 * 2 * D * 2, 2 * D, S, nullptr, 0, 0, nullptr,
-                       n, (int)(2 * D), (int)D, XEMA_EPI_BIAS);
+                       n, (int)(2 * D), (int)D, XEMA_EPI_BIAS, "KV", ci);
       if (rc) return rc;
       Op o{};
       o.kind = OP_ROPE;
+      tag(o, "KROPE", ci, 12.0 * Bd * n * Dd, 4.0 * Bd * n * Dd + 4.0 * n * c.head_dim);
       o.rope_x = kv + r0 * 2 * D * 2; o.rope_ld = 2 * D; o.rope_batch_rows = S; o.rope_g = w.g_k;
       o.pos0 = (int)r0; o.rows = n;
       plan->ops.push_back(o);
@@ -303,22 +321,26 @@ int xema_plan_bind(xema_plan* plan, void* arena_dev, uint64_t arena_bytes, const
       uint8_t* o_t = at("o", l, ci);
       float* lse = reinterpret_cast<float*>(at("lse", l, ci));
       if (!h1b || !q || !o_t || !lse) return XEMA_EINVAL;
-      ln_op(hid + r0 * D * 2, 0, h1b, n, 1);
-      int rc = gemm_op(h1b, D, n, w_qkv, D, b_qkv, q, D, n, nullptr, 0, 0, nullptr, n, (int)D, (int)D, XEMA_EPI_BIAS);
+      ln_op(hid + r0 * D * 2, 0, h1b, n, 1, "LN1B", ci);
+      int rc = gemm_op(h1b, D, n, w_qkv, D, b_qkv, q, D, n, nullptr, 0, 0, nullptr, n, (int)D, (int)D, XEMA_EPI_BIAS,
+                       "Q", ci);
       if (rc) return rc;
       Op o{};
       o.kind = OP_ROPE;
+      tag(o, "QROPE", ci, 12.0 * Bd * n * Dd, 4.0 * Bd * n * Dd + 4.0 * n * c.head_dim);
       o.rope_x = q; o.rope_ld = D; o.rope_batch_rows = n; o.rope_g = w.g_q; o.pos0 = (int)r0; o.rows = n;
       plan->ops.push_back(o);
       Op a{};
       a.kind = OP_ATTN;
+      // q and o once, k and v once per launch, lse
+      tag(a, "ATTN", ci, 4.0 * Bd * n * Sd * Dd, 4.0 * Bd * n * Dd + 4.0 * Bd * Sd * Dd + 4.0 * Bd * c.heads * n);
       a.attn.o = o_t; a.attn.lse = lse; a.attn.batch = c.batch; a.attn.rows = n; a.attn.keys = (int)S;
       a.attn.heads = c.heads; a.attn.head_dim = c.head_dim; a.attn.status = status;
       rc = attn_prepare(&a.attn, q, D, n, kv, kv + D * 2, 2 * D, S);
       if (rc) return rc;
       plan->ops.push_back(a);
       rc = gemm_op(o_t, D, n, w.w_o, D, w.b_o, res + r0 * D * 4, D, S, hid + r0 * D * 2, D, S, mod + 2 * D, n, (int)D,
-                   (int)D, XEMA_EPI_GATE_RES_F32);
+                   (int)D, XEMA_EPI_GATE_RES_F32, "PROJ", ci);
       if (rc) return rc;
     }
     // phase C: feed-forward of every chunk
@@ -328,12 +350,12 @@ int xema_plan_bind(xema_plan* plan, void* arena_dev, uint64_t arena_bytes, const
       uint8_t* h2 = at("h2", l, ci);
       uint8_t* g = at("g", l, ci);
       if (!h2 || !g) return XEMA_EINVAL;
-      ln_op(res + r0 * D * 4, 1, h2, n, 2);
+      ln_op(res + r0 * D * 4, 1, h2, n, 2, "LN2", ci);
       int rc = gemm_op(h2, D, n, w.w_1, D, w.b_1, g, F, n, nullptr, 0, 0, nullptr, n, (int)F, (int)D,
-                       XEMA_EPI_BIAS_GELU);
+                       XEMA_EPI_BIAS_GELU, "FFN1", ci);
       if (rc) return rc;
       rc = gemm_op(g, F, n, w.w_2, F, w.b_2, hid_next + r0 * D * 2, D, S, res + r0 * D * 4, D, S, mod + 5 * D, n,
-                   (int)D, (int)F, XEMA_EPI_GATE_RES_BF16);
+                   (int)D, (int)F, XEMA_EPI_GATE_RES_BF16, "FFN2", ci);
       if (rc) return rc;
     }
   }
@@ -345,16 +367,35 @@ int xema_plan_bind(xema_plan* plan, void* arena_dev, uint64_t arena_bytes, const
 int xema_block_forward(const xema_plan* plan, void* stream) {
   if (!plan) return XEMA_EINVAL;
   if (plan->cfg.n_blocks != 1) return XEMA_ESTATE;
-  return run_ops(plan, plan->ops.size(), stream);
+  return run_ops(plan, 0, plan->ops.size(), stream);
 }
 
 int xema_step_forward(const xema_plan* plan, void* stream) {
   if (!plan) return XEMA_EINVAL;
-  return run_ops(plan, plan->ops.size(), stream);
+  return run_ops(plan, 0, plan->ops.size(), stream);
 }
 
 int xema_forward_prefix(const xema_plan* plan, uint32_t n_logical_ops, void* stream) {
-  return run_ops(plan, n_logical_ops, stream);
+  return run_ops(plan, 0, n_logical_ops, stream);
+}
+
+int xema_forward_range(const xema_plan* plan, uint32_t first_op, uint32_t end_op, void* stream) {
+  if (first_op > end_op) return XEMA_EINVAL;
+  return run_ops(plan, first_op, end_op, stream);
+}
+
+int xema_plan_op(const xema_plan* plan, uint32_t i, char* name8, int32_t* block, int32_t* chunk, double* flops,
+                 double* bytes) {
+  if (!plan) return XEMA_EINVAL;
+  if (!plan->bound) return XEMA_ESTATE;
+  if (i >= plan->ops.size()) return XEMA_EINVAL;
+  const Op& o = plan->ops[i];
+  if (name8) std::memcpy(name8, o.name, 8);
+  if (block) *block = o.block;
+  if (chunk) *chunk = o.chunk;
+  if (flops) *flops = o.flops;
+  if (bytes) *bytes = o.bytes;
+  return XEMA_OK;
 }
 
 int xema_plan_launch_count(const xema_plan* plan) {
