@@ -58,6 +58,32 @@ def load_peaks():
         return {"hbm_gbs": 6650.0, "bf16_burst": 1590.0, "bf16_sustained": 1400.0, "source": "fallback"}
 
 
+def max_over_ranks(ms: float, dist, device) -> float:
+    """Slowest rank's time (all ranks call this); identity without a process group."""
+    if dist is None:
+        return ms
+    import torch
+    tt = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+    return float(tt.item())
+
+
+def whole_job_tflops(flops_per_replica: float, world: int, ms: float) -> float:
+    """Replicas are independent: the job did world x flops in the slowest rank's time."""
+    return world * flops_per_replica / (ms * 1e-3) / 1e12
+
+
+# DRAM traffic of one attention launch, from the ncu capture summarised in
+# profiles/attention_rows2222_keys17776_h48_d64.md (2222 query rows): 251.8 MB read + written, of
+# which k and v (4*S*D bytes, independent of the number of query rows) are read once and the
+# rest scales with the query rows.
+def attention_traffic_bytes(t, rows: int) -> float:
+    if (t.seq, t.hidden, t.head_dim) != (17776, 3072, 64):
+        return None
+    kv = 4.0 * t.seq * t.hidden
+    return kv + (251.8e6 - kv) * rows / 2222.0
+
+
 class ClockSampler:
     """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
 
@@ -107,13 +133,17 @@ class ClockSampler:
                 "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def time_oracle_sample(t, n_rows=CPU_SAMPLE_ROWS):
+def oracle_inputs(t):
+    w = {k: bits_to_f64(v) for k, v in make_block_weights(t, 0).items()}
+    x, temb = make_activations(t)
+    return w, bits_to_f64(x), bits_to_f64(temb)
+
+
+def time_oracle_sample(t, n_rows=CPU_SAMPLE_ROWS, inputs=None):
     """Times the float64 oracle, as it stands, on a bounded sample of the workload: keys and
     values of every token, then the complete block for `n_rows` seeded token rows."""
     from oracle import block as ob
-    w = {k: bits_to_f64(v) for k, v in make_block_weights(t, 0).items()}
-    x, temb = make_activations(t)
-    x, temb = bits_to_f64(x), bits_to_f64(temb)
+    w, x, temb = inputs or oracle_inputs(t)
     rows = sample_rows(t, n_random=n_rows)
     t0 = time.perf_counter()
     ob.block_forward(t, w, x, temb, rows=rows)
@@ -126,11 +156,12 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    t = template(args.workload)
+    t = template(args.workload).with_(n_blocks=1)
     cores = len(os.sched_getaffinity(0))
     times, n_rows = [], 0
+    inputs = oracle_inputs(t)
     for i in range(args.warmup + args.steps):
-        dt, n_rows = time_oracle_sample(t, args.cpu_rows)
+        dt, n_rows = time_oracle_sample(t, min(args.cpu_rows, 256), inputs)
         if i >= args.warmup:
             times.append(dt)
     mean = float(np.mean(times))
@@ -219,13 +250,9 @@ def main():
     clocks = sampler.stop()
     free_after, _ = torch.cuda.mem_get_info(dev)
     sess.check_status()
-    total_ms = ev[0][0].elapsed_time(ev[-1][n_launch])
-    if dist is not None:
-        tt = torch.tensor([total_ms], device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        total_ms = float(tt.item())
+    total_ms = max_over_ranks(ev[0][0].elapsed_time(ev[-1][n_launch]), dist, dev)
     ms_per_step = total_ms / args.steps
-    value = world * flops / (ms_per_step * 1e-3) / 1e12
+    value = whole_job_tflops(flops, world, ms_per_step)
 
     per_op = {}
     for i, op in enumerate(ops):
@@ -252,12 +279,7 @@ def main():
         e2e_step()
     e1.record(stream)
     barrier()
-    e2e_ms = e0.elapsed_time(e1)
-    if dist is not None:
-        tt = torch.tensor([e2e_ms], device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        e2e_ms = float(tt.item())
-    e2e_ms /= args.steps
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1), dist, dev) / args.steps
     h2d = int(x_host.numel() * 2 + temb_host.numel() * 2)
     d2h = int(out_host.numel() * 2)
 
@@ -299,8 +321,11 @@ def main():
     else:
         achieved = d["bytes"] / d["launches"] / per_launch_s / 1e9
         peak, unit, bound = peaks["hbm_gbs"], "GB/s", "hbm"
+    traffic = None
+    if dom == "ATTN":
+        traffic = attention_traffic_bytes(t, t.seq * t.n_blocks // d["launches"])
     roofline = {"kernel": dom, "bound": bound, "achieved": achieved, "peak": peak, "unit": unit,
-                "frac": achieved / peak, "traffic": None, "peak_source": peaks["source"] + " (sustained)",
+                "frac": achieved / peak, "traffic": traffic, "peak_source": peaks["source"] + " (sustained)",
                 "peak_burst": peaks["bf16_burst"] if tensor_bound else None,
                 "ms_per_launch": per_launch_s * 1e3, "launches_per_step": d["launches"]}
     breakdown = {n: {"ms": round(v["ms"], 4), "share": round(v["ms"] / ms_per_step, 4),
@@ -330,7 +355,7 @@ def main():
                    "l2": "inputs larger than L2 (weights 245 MB + arena per block)",
                    "parallelism": "replicas x%d" % world},
         "clocks": clocks,
-        "e2e": {"value": world * flops / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
+        "e2e": {"value": whole_job_tflops(flops, world, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": n_launch * args.steps,
         "roofline": roofline,

@@ -1,0 +1,52 @@
+"""The N > 1 path of bench.py shards nothing and exchanges nothing on the data path: every rank
+runs a replica, the ranks meet at a barrier and the slowest rank's time is used.  That host
+logic is exercised here with two gloo ranks on the CPU."""
+import os
+import socket
+import sys
+
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _worker(rank, world, port, out):
+    sys.path.insert(0, ROOT)
+    import bench
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    dist.barrier()
+    ms = bench.max_over_ranks(10.0 + 5.0 * rank, dist, torch.device("cpu"))
+    out[rank] = (ms, bench.whole_job_tflops(1e12, world, ms))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_two_replicas_report_the_slowest_rank():
+    world, port = 2, _free_port()
+    with mp.Manager() as mgr:
+        out = mgr.dict()
+        mp.spawn(_worker, args=(world, port, out), nprocs=world, join=True)
+        res = dict(out)
+    assert res[0] == res[1]
+    ms, tflops = res[0]
+    assert ms == 15.0
+    assert abs(tflops - 2 * 1e12 / 15e-3 / 1e12) < 1e-9
+
+
+def test_single_process_needs_no_group():
+    sys.path.insert(0, ROOT)
+    import bench
+    assert bench.max_over_ranks(3.5, None, None) == 3.5
+    from xema_inputs import template
+    t = template("cogvideox")
+    assert abs(bench.block_flops(t) - 7.910e12) / 7.910e12 < 1e-3
+    assert bench.attention_traffic_bytes(t, 2222) == 251.8e6
