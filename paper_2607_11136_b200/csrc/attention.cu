@@ -9,7 +9,9 @@
 //   warps 2-5 softmax: thread = query row.  Read S from TMEM, running max / sum in the exp2
 //             domain, write P (bf16) into shared memory in the 128-byte-swizzled K-major
 //             layout the MMA reads, rescale O in TMEM when the running max moved, and at
-//             the end normalise O and store it.
+//             the end normalise O and store it.  The score row is held in registers, so the
+//             S buffer is handed back right after the load and S(j+1) = Q K(j+1)^T runs while
+//             the exponentials of block j are evaluated.
 // Every decision is taken per row (the running max only moves when it grows by more than 2^8
 // in the exp2 domain; multiplying the other rows by exactly 1 changes nothing), keys are
 // always visited from key 0 in blocks of 128, and nothing is split or reduced across CTAs, so
@@ -68,7 +70,8 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   uint64_t* s_full = bars + 9;
   uint64_t* p_full = bars + 10;
   uint64_t* pv_done = bars + 11;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 12);
+  uint64_t* s_free = bars + 12;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 13);
   volatile uint32_t* abort_flag = tmem_slot + 1;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -91,6 +94,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     }
     mbar_init(s_full, 1);
     mbar_init(p_full, 4);
+    mbar_init(s_free, 4);
     mbar_init(pv_done, 1);
     *abort_flag = 0;
     fence_mbar_init();
@@ -179,10 +183,14 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       for (int j = 0; ok && j < n_kv; ++j) {
         const int st = j % ATT_KV_STAGES;
         const uint32_t ph = (uint32_t)(j / ATT_KV_STAGES) & 1u;
-        // softmax has read all of S(j) and written P(j)
+        // as soon as the softmax warps hold S(j) in registers, S(j+1) may overwrite it
+        if (j + 1 < n_kv) {
+          if (!(ok = mbar_wait(s_free, j & 1, abort_flag))) break;
+          tc_fence_after();
+          if (!(ok = issue_s(j + 1))) break;
+        }
+        // P(j) is in shared memory (and O has been rescaled if the max moved)
         if (!(ok = mbar_wait(p_full, j & 1, abort_flag))) break;
-        tc_fence_after();
-        if (j + 1 < n_kv && !(ok = issue_s(j + 1))) break;
         if (!(ok = mbar_wait(&v_full[st], ph, abort_flag))) break;
         tc_fence_after();
         const uint32_t v_addr = smem_u32(smem + Cfg::OFF_V + st * Cfg::TILE_BYTES);
@@ -212,25 +220,50 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      const int valid = min(ATT_BN, p.keys - j * ATT_BN);   // < 128 only in the last block
-      // pass 1: row max of the raw scores
-      float m_blk = -INFINITY;
-#pragma unroll 1
-      for (int ch = 0; ch < ATT_BN / 32; ++ch) {
-        uint32_t s[32];
-        tmem_ld32(tmem_s + lane_sel + ch * 32, s);
-        tmem_ld_wait();
+      // the whole score row of this thread into registers, then hand the TMEM buffer back
+      float s[ATT_BN];
 #pragma unroll
-        for (int t = 0; t < 32; ++t) {
-          const float v = (ch * 32 + t < valid) ? __uint_as_float(s[t]) : -INFINITY;
-          m_blk = fmaxf(m_blk, v);
-        }
+      for (int ch = 0; ch < ATT_BN / 32; ++ch)
+        tmem_ld32(tmem_s + lane_sel + ch * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[ch * 32]));
+      tmem_ld_wait();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(s_free);
+      // keys past the end exist only in the last block
+      const int valid = p.keys - j * ATT_BN;
+      if (valid < ATT_BN) {
+#pragma unroll
+        for (int t = 0; t < ATT_BN; ++t)
+          if (t >= valid) s[t] = -INFINITY;
       }
+      // row max: independent partial maxima, three-input max
+      float mx[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) mx[u] = max3(s[16 * u], s[16 * u + 1], s[16 * u + 2]);
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+#pragma unroll
+        for (int t = 3; t < 15; t += 2) mx[u] = max3(mx[u], s[16 * u + t], s[16 * u + t + 1]);
+        mx[u] = fmaxf(mx[u], s[16 * u + 15]);
+      }
+      const float m_blk = fmaxf(max3(mx[0], mx[1], mx[2]), max3(max3(mx[3], mx[4], mx[5]), mx[6], mx[7]));
       // the running max moves only when it grows by more than 2^8 (exp2 domain); per row
       float m_new = m_run;
       if (j == 0 || (m_blk - m_run) * p.scale_log2 > 8.f) m_new = m_blk;
       const float alpha = (j == 0 || m_new == m_run) ? 1.f : ex2_approx((m_run - m_new) * p.scale_log2);
       const float neg_m = -m_new * p.scale_log2;
+      // p = exp2(s * c - m * c); row sum in four independent partial sums; pack to bf16
+      float ls[4] = {0.f, 0.f, 0.f, 0.f};
+      uint32_t pk[ATT_BN / 2];
+#pragma unroll
+      for (int t = 0; t < ATT_BN; t += 2) {
+        const float e0 = ex2_approx(fmaf(s[t], p.scale_log2, neg_m));
+        const float e1 = ex2_approx(fmaf(s[t + 1], p.scale_log2, neg_m));
+        ls[(t >> 1) & 3] += e0 + e1;
+        pk[t >> 1] = pack_bf16x2(e0, e1);
+      }
+      l_run = fmaf(l_run, alpha, (ls[0] + ls[1]) + (ls[2] + ls[3]));
+      m_run = m_new;
       // P(j) overwrites the buffer PV(j-1) reads, and O must be at rest before it is rescaled
       if (j > 0) {
         ok = mbar_wait(pv_done, (j - 1) & 1, abort_flag);
@@ -238,31 +271,12 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         if (!ok) break;
         tc_fence_after();
       }
-      // pass 2: p = exp2(s * c - m * c), row sum, bf16 P into swizzled shared memory
-      float l_blk = 0.f;
-#pragma unroll 1
-      for (int ch = 0; ch < ATT_BN / 32; ++ch) {
-        uint32_t s[32];
-        tmem_ld32(tmem_s + lane_sel + ch * 32, s);
-        tmem_ld_wait();
-        float pv[32];
 #pragma unroll
-        for (int t = 0; t < 32; ++t) {
-          const float e = ex2_approx(fmaf(__uint_as_float(s[t]), p.scale_log2, neg_m));
-          pv[t] = (ch * 32 + t < valid) ? e : 0.f;
-          l_blk += pv[t];
-        }
-        uint8_t* atom_row = p_row + (ch / 2) * ATOM_BYTES;
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const int chunk16 = (ch & 1) * 4 + q;             // 16-byte chunk inside the 128-byte row
-          uint4 w = make_uint4(pack_bf16x2(pv[8 * q + 0], pv[8 * q + 1]), pack_bf16x2(pv[8 * q + 2], pv[8 * q + 3]),
-                               pack_bf16x2(pv[8 * q + 4], pv[8 * q + 5]), pack_bf16x2(pv[8 * q + 6], pv[8 * q + 7]));
-          *reinterpret_cast<uint4*>(atom_row + ((chunk16 ^ swz) << 4)) = w;
-        }
+      for (int c16 = 0; c16 < ATT_BN / 8; ++c16) {          // 16-byte chunks of the 256-byte P row
+        uint8_t* atom_row = p_row + (c16 / 8) * ATOM_BYTES;
+        *reinterpret_cast<uint4*>(atom_row + (((c16 & 7) ^ swz) << 4)) =
+            make_uint4(pk[4 * c16], pk[4 * c16 + 1], pk[4 * c16 + 2], pk[4 * c16 + 3]);
       }
-      l_run = fmaf(l_run, alpha, l_blk);
-      m_run = m_new;
       // rescale O where the max moved (rows that kept their max multiply by exactly 1)
       if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
 #pragma unroll 1
