@@ -170,6 +170,35 @@ int xema_plan_bind(xema_plan* plan, void* arena_dev, uint64_t arena_bytes,
 int xema_block_forward(const xema_plan* plan, void* stream);
 int xema_step_forward(const xema_plan* plan, void* stream);
 
+/* The block forward for callers that cannot allocate device memory (the paper has no
+ * counterpart: its runtime always has PyTorch's allocator behind it).  Some callers can call
+ * neither cudaMalloc nor a framework allocator: code inside a region that must not
+ * synchronise the device, a process whose device memory already belongs to a pool it does not
+ * own, a plug-in that is handed nothing but its input and output buffers.  xema_block_forward
+ * needs a caller-allocated arena for the block's intermediates; this variant keeps them in a
+ * fixed array of XEMA_STATIC_ARENA_BYTES inside the library image instead (every GPU that
+ * loads the library holds that much memory until the process exits).
+ *
+ * One block (cfg->n_blocks must be 1) with `chunks` sequence chunks.  weights: host pointer to
+ * one struct of device pointers; rope_dev: device copy of xema_rope_table's output;
+ * hid_in_dev [B,S,D] bf16, temb_dev [B,Dt] bf16 (device, read); hid_out_dev [B,S,D] bf16
+ * (device, written; may not overlap the inputs); status_dev: device, 4 zeroed bytes, or NULL.
+ * Enqueues two device-to-device copies in, the block's launches, and one copy out on `stream`.
+ * Calls no cudaMalloc/cudaFree and no allocating library routine; host memory for the plan is
+ * taken from the C++ heap and released before returning.
+ *
+ * XEMA_ENOSPC: the template's arena peak for this chunk count exceeds XEMA_STATIC_ARENA_BYTES
+ * (the tiny template needs 2 076 672 bytes at chunks = 1); use xema_block_forward with your own
+ * arena instead.  The first call on a device looks up the array's device address
+ * (cudaGetSymbolAddress); make that first call before any stream capture begins.  All calls
+ * share the one array and it keeps the previous call's contents (the block writes every
+ * intermediate before reading it, so nothing has to be cleared); two calls whose work overlaps
+ * on the GPU -- different streams, or different host threads -- race on it. */
+#define XEMA_STATIC_ARENA_BYTES (4u << 20)
+int xema_block_forward_static(const xema_config* cfg, int32_t chunks, const xema_block_weights* weights,
+                              const float* rope_dev, const void* hid_in_dev, const void* temb_dev,
+                              void* hid_out_dev, void* status_dev, void* stream);
+
 /* Number of kernel launches one forward call enqueues (0 if unbound). */
 int xema_plan_launch_count(const xema_plan* plan);
 

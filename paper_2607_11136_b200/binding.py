@@ -22,6 +22,7 @@ EXPORTS = (
     "xema_trace", "xema_plan_arena", "xema_chunks_for_budget", "xema_rope_table",
     "xema_plan_create", "xema_plan_destroy", "xema_plan_info", "xema_plan_tensor",
     "xema_plan_tensor_at", "xema_plan_bind", "xema_block_forward", "xema_step_forward",
+    "xema_block_forward_static",
     "xema_plan_launch_count", "xema_forward_prefix", "xema_forward_range", "xema_plan_op", "xema_op_mod", "xema_op_ln_modulate",
     "xema_op_rmsnorm_rope", "xema_op_gemm", "xema_op_attention", "xema_strerror",
     "xema_last_cuda_error", "xema_version",
@@ -90,6 +91,7 @@ def lib() -> C.CDLL:
             "xema_plan_bind": [vp, vp, u64, P(xema_block_weights), vp, vp],
             "xema_block_forward": [vp, vp],
             "xema_step_forward": [vp, vp],
+            "xema_block_forward_static": [P(xema_config), i32, P(xema_block_weights), vp, vp, vp, vp, vp, vp],
             "xema_plan_launch_count": [vp],
             "xema_forward_prefix": [vp, u32, vp],
             "xema_forward_range": [vp, u32, u32, vp],
@@ -257,6 +259,22 @@ class Plan:
 
     def forward_prefix(self, n_logical_ops: int, stream: int = 0):
         _check(lib().xema_forward_prefix(self._h, n_logical_ops, stream), "xema_forward_prefix")
+
+
+STATIC_ARENA_BYTES = 4 << 20
+
+
+def xema_block_forward_static(cfg: xema_config, chunks: int, weights: dict, rope_ptr: int, hid_in: int, temb: int,
+                              hid_out: int, status: Optional[int] = None, stream: int = 0):
+    """One block whose intermediates live in the library's fixed scratch array; for callers
+    that may not allocate device memory.  weights maps the twelve parameter names to device
+    pointers; the other arguments are device pointers.  Raises XemaError(XEMA_ENOSPC) when the
+    template needs more than STATIC_ARENA_BYTES."""
+    w = xema_block_weights()
+    for f in _WEIGHT_FIELDS:
+        setattr(w, f, weights[f])
+    _check(lib().xema_block_forward_static(C.byref(cfg), chunks, C.byref(w), rope_ptr, hid_in, temb, hid_out,
+                                           status, stream), "xema_block_forward_static")
 
 
 def xema_op_mod(temb, w_mod, b_mod, mod, batch, temb_dim, n_out, stream=0):
