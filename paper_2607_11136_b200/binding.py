@@ -12,7 +12,7 @@ from typing import Optional, Sequence
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libxema.so")
+LIB_PATH = os.environ.get("XEMA_LIB") or os.path.join(_HERE, "libxema.so")
 
 XEMA_OK, XEMA_EINVAL, XEMA_ENOSPC, XEMA_EBUDGET = 0, -1, -2, -3
 XEMA_EALIGN, XEMA_ECUDA, XEMA_ETIMEOUT, XEMA_ESTATE = -4, -5, -6, -7

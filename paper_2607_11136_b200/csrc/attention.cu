@@ -7,9 +7,10 @@
 //   warp 1    owns TMEM; one thread issues S = Q K^T (TMEM, 128 fp32 columns) and
 //             O += P V (TMEM, dh fp32 columns)
 //   warps 2-5 softmax: thread = query row.  Read S from TMEM, running max / sum in the exp2
-//             domain, write P (bf16) into shared memory in the 128-byte-swizzled K-major
-//             layout the MMA reads, rescale O in TMEM when the running max moved, and at
-//             the end normalise O and store it.  The score row is held in registers, so the
+//             domain, write P (bf16, two per column) back into TMEM where the second MMA reads
+//             it as its A operand (shared memory carries only Q, K and V: its bandwidth, not
+//             the tensor pipe, bounds this kernel), rescale O in TMEM when the running max
+//             moved, and at the end normalise O and store it.  The score row is held in registers, so the
 //             S buffer is handed back right after the load and S(j+1) = Q K(j+1)^T runs while
 //             the exponentials of block j are evaluated.
 // Every decision is taken per row (the running max only moves when it grows by more than 2^8
@@ -27,23 +28,35 @@ using namespace sm100;
 constexpr int ATT_BM = 128;      // query rows per CTA
 constexpr int ATT_BN = 128;      // keys per block
 constexpr int ATT_THREADS = 192;
-constexpr int ATT_KV_STAGES = 2;
 constexpr int ATOM_BYTES = 128 * 128;   // 128 rows x 64 bf16, one swizzled column block
+// share of the exponentials evaluated as a polynomial on the FMA pipe instead of the MUFU
+#ifndef XEMA_ATT_POLY_NUM
+#define XEMA_ATT_POLY_NUM 1
+#endif
+#ifndef XEMA_ATT_POLY_DEN
+#define XEMA_ATT_POLY_DEN 4
+#endif
+constexpr int POLY_NUM = XEMA_ATT_POLY_NUM, POLY_DEN = XEMA_ATT_POLY_DEN;
 
 template <int DH>
 struct AttnCfg {
   static constexpr int ATOMS = DH / 64;                      // 64-wide column blocks per tile
   static constexpr int TILE_BYTES = ATOMS * ATOM_BYTES;      // Q, K or V tile
-  static constexpr int P_BYTES = (ATT_BN / 64) * ATOM_BYTES;
+  static constexpr int KV_STAGES = (DH == 64) ? 3 : 2;
   static constexpr int OFF_Q = 0;
   static constexpr int OFF_K = OFF_Q + TILE_BYTES;
-  static constexpr int OFF_V = OFF_K + ATT_KV_STAGES * TILE_BYTES;
-  static constexpr int OFF_P = OFF_V + ATT_KV_STAGES * TILE_BYTES;
-  static constexpr int OFF_BAR = OFF_P + P_BYTES;
+  static constexpr int OFF_V = OFF_K + KV_STAGES * TILE_BYTES;
+  static constexpr int OFF_BAR = OFF_V + KV_STAGES * TILE_BYTES;
   static constexpr int SMEM_BYTES = OFF_BAR + 256;
-  static constexpr int TMEM_COLS = 256;                      // S: [0,128), O: [128, 128+DH)
-  static constexpr int TMEM_O = 128;
+  // TMEM columns: S fp32 [0,128); P bf16, two per column [128,192); O fp32 [192, 192+DH)
+  static constexpr int TMEM_P = 128;
+  static constexpr int TMEM_O = 192;
+  static constexpr int TMEM_COLS = (DH == 64) ? 256 : 512;
+#ifdef XEMA_DBG_ONE_CTA
+  static constexpr int MIN_CTAS = 1;
+#else
   static constexpr int MIN_CTAS = (DH == 64) ? 2 : 1;
+#endif
 };
 
 struct AttnParams {
@@ -63,15 +76,15 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   extern __shared__ __align__(1024) uint8_t smem[];
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + Cfg::OFF_BAR);
   uint64_t* q_full = bars + 0;
-  uint64_t* k_full = bars + 1;    // [2]
-  uint64_t* k_empty = bars + 3;   // [2]
-  uint64_t* v_full = bars + 5;    // [2]
-  uint64_t* v_empty = bars + 7;   // [2]
-  uint64_t* s_full = bars + 9;
-  uint64_t* p_full = bars + 10;
-  uint64_t* pv_done = bars + 11;
-  uint64_t* s_free = bars + 12;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 13);
+  uint64_t* k_full = bars + 1;    // [KV_STAGES <= 3]
+  uint64_t* k_empty = bars + 4;
+  uint64_t* v_full = bars + 7;
+  uint64_t* v_empty = bars + 10;
+  uint64_t* s_full = bars + 13;
+  uint64_t* p_full = bars + 14;
+  uint64_t* pv_done = bars + 15;
+  uint64_t* s_free = bars + 16;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 17);
   volatile uint32_t* abort_flag = tmem_slot + 1;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -86,7 +99,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 
   if (threadIdx.x == 0) {
     mbar_init(q_full, 1);
-    for (int s = 0; s < ATT_KV_STAGES; ++s) {
+    for (int s = 0; s < Cfg::KV_STAGES; ++s) {
       mbar_init(&k_full[s], 1);
       mbar_init(&k_empty[s], 1);
       mbar_init(&v_full[s], 1);
@@ -111,6 +124,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   const uint32_t tmem_s = tmem_base;
+  const uint32_t tmem_p = tmem_base + Cfg::TMEM_P;
   const uint32_t tmem_o = tmem_base + Cfg::TMEM_O;
 
   if (warp == 0) {
@@ -123,8 +137,8 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         tma_load_3d(smem + Cfg::OFF_Q + a * ATOM_BYTES, &map_q, q_full, h * DH + a * 64, qt * ATT_BM, b);
       int k_issued = 0, v_issued = 0;
       for (int j = 0; j < n_kv; ++j) {
-        const int st = j % ATT_KV_STAGES;
-        const uint32_t ph = (uint32_t)(j / ATT_KV_STAGES) & 1u;
+        const int st = j % Cfg::KV_STAGES;
+        const uint32_t ph = (uint32_t)(j / Cfg::KV_STAGES) & 1u;
         if (!(ok = mbar_wait(&k_empty[st], ph ^ 1, abort_flag))) break;
         mbar_expect_tx(&k_full[st], Cfg::TILE_BYTES);
 #pragma unroll
@@ -145,13 +159,13 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         // fill of each stage; older fills were consumed before their stage was reused)
         volatile uint32_t dummy = 0;
         mbar_wait(q_full, 0, &dummy);
-        for (int j = max(0, k_issued - ATT_KV_STAGES); j < k_issued; ++j) {
+        for (int j = max(0, k_issued - Cfg::KV_STAGES); j < k_issued; ++j) {
           dummy = 0;
-          mbar_wait(&k_full[j % ATT_KV_STAGES], (uint32_t)(j / ATT_KV_STAGES) & 1u, &dummy);
+          mbar_wait(&k_full[j % Cfg::KV_STAGES], (uint32_t)(j / Cfg::KV_STAGES) & 1u, &dummy);
         }
-        for (int j = max(0, v_issued - ATT_KV_STAGES); j < v_issued; ++j) {
+        for (int j = max(0, v_issued - Cfg::KV_STAGES); j < v_issued; ++j) {
           dummy = 0;
-          mbar_wait(&v_full[j % ATT_KV_STAGES], (uint32_t)(j / ATT_KV_STAGES) & 1u, &dummy);
+          mbar_wait(&v_full[j % Cfg::KV_STAGES], (uint32_t)(j / Cfg::KV_STAGES) & 1u, &dummy);
         }
       }
     }
@@ -161,10 +175,9 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       constexpr uint32_t idesc_s = idesc_bf16_f32(ATT_BM, ATT_BN, false, false);   // S = Q K^T
       constexpr uint32_t idesc_o = idesc_bf16_f32(ATT_BM, DH, false, true);        // O = P V, V is N-major
       const uint32_t q_addr = smem_u32(smem + Cfg::OFF_Q);
-      const uint32_t p_addr = smem_u32(smem + Cfg::OFF_P);
       auto issue_s = [&](int j) -> bool {
-        const int st = j % ATT_KV_STAGES;
-        const uint32_t ph = (uint32_t)(j / ATT_KV_STAGES) & 1u;
+        const int st = j % Cfg::KV_STAGES;
+        const uint32_t ph = (uint32_t)(j / Cfg::KV_STAGES) & 1u;
         if (!mbar_wait(&k_full[st], ph, abort_flag)) return false;
         tc_fence_after();
         const uint32_t k_addr = smem_u32(smem + Cfg::OFF_K + st * Cfg::TILE_BYTES);
@@ -181,8 +194,8 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       bool ok = mbar_wait(q_full, 0, abort_flag);
       if (ok) ok = issue_s(0);
       for (int j = 0; ok && j < n_kv; ++j) {
-        const int st = j % ATT_KV_STAGES;
-        const uint32_t ph = (uint32_t)(j / ATT_KV_STAGES) & 1u;
+        const int st = j % Cfg::KV_STAGES;
+        const uint32_t ph = (uint32_t)(j / Cfg::KV_STAGES) & 1u;
         // as soon as the softmax warps hold S(j) in registers, S(j+1) may overwrite it
         if (j + 1 < n_kv) {
           if (!(ok = mbar_wait(s_free, j & 1, abort_flag))) break;
@@ -196,11 +209,11 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         const uint32_t v_addr = smem_u32(smem + Cfg::OFF_V + st * Cfg::TILE_BYTES);
 #pragma unroll
         for (int kk = 0; kk < ATT_BN / 16; ++kk) {
-          const uint64_t da = smem_desc_sw128(p_addr + (kk / 4) * ATOM_BYTES + (kk % 4) * 32, 16, 1024);
+          // P from TMEM: 16 keys = 8 packed columns per instruction.
           // V tile: rows = keys (the MMA's K), 64 dh per 128-byte row; 16 keys = 2048 bytes;
           // the second 64-wide dh block (dh = 128) starts one atom further
           const uint64_t db = smem_desc_sw128(v_addr + kk * 2048, ATOM_BYTES, 1024);
-          mma_ss(tmem_o, da, db, idesc_o, (j | kk) != 0);
+          mma_ts(tmem_o, tmem_p + kk * 8, db, idesc_o, (j | kk) != 0);
         }
         mma_commit(&v_empty[st]);
         mma_commit(pv_done);
@@ -211,8 +224,6 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     const int quad = warp & 3;
     const int r = quad * 32 + lane;                       // query row inside the tile = TMEM lane
     const uint32_t lane_sel = (uint32_t)(quad * 32) << 16;
-    uint8_t* p_row = smem + Cfg::OFF_P + r * 128;
-    const int swz = r & 7;
     float m_run = -INFINITY, l_run = 0.f;
     bool ok = true;
     for (int j = 0; j < n_kv; ++j) {
@@ -252,15 +263,43 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       if (j == 0 || (m_blk - m_run) * p.scale_log2 > 8.f) m_new = m_blk;
       const float alpha = (j == 0 || m_new == m_run) ? 1.f : ex2_approx((m_run - m_new) * p.scale_log2);
       const float neg_m = -m_new * p.scale_log2;
-      // p = exp2(s * c - m * c); row sum in four independent partial sums; pack to bf16
-      float ls[4] = {0.f, 0.f, 0.f, 0.f};
+      // p = exp2(s * c - m * c) on pairs of columns with packed fp32x2 arithmetic; POLY_NUM of
+      // every POLY_DEN pairs (fixed column positions) evaluate 2^x as a polynomial on the FMA
+      // pipe, the rest on the MUFU; row sum in four independent packed partial sums
+      const uint64_t c2 = pack_f32x2(p.scale_log2, p.scale_log2);
+      const uint64_t nm2 = pack_f32x2(neg_m, neg_m);
+      uint64_t ls2[4] = {0ull, 0ull, 0ull, 0ull};
       uint32_t pk[ATT_BN / 2];
 #pragma unroll
       for (int t = 0; t < ATT_BN; t += 2) {
-        const float e0 = ex2_approx(fmaf(s[t], p.scale_log2, neg_m));
-        const float e1 = ex2_approx(fmaf(s[t + 1], p.scale_log2, neg_m));
-        ls[(t >> 1) & 3] += e0 + e1;
-        pk[t >> 1] = pack_bf16x2(e0, e1);
+        const int pair = t >> 1;
+        uint64_t e2 = fma_f32x2(pack_f32x2(s[t], s[t + 1]), c2, nm2);
+        float e0, e1;
+        if ((pair % POLY_DEN) < POLY_NUM) {
+          e2 = exp2_poly_f32x2(e2);
+          unpack_f32x2(e2, e0, e1);
+        } else {
+          unpack_f32x2(e2, e0, e1);
+#ifdef XEMA_DBG_NOEXP
+          e0 = e0 * 0.001f + 1.f;
+          e1 = e1 * 0.001f + 1.f;
+#else
+          e0 = ex2_approx(e0);
+          e1 = ex2_approx(e1);
+#endif
+          e2 = pack_f32x2(e0, e1);
+        }
+        ls2[pair & 3] = add_f32x2(ls2[pair & 3], e2);
+        pk[pair] = pack_bf16x2(e0, e1);
+      }
+      float ls[4];
+      {
+        float a, b;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          unpack_f32x2(ls2[u], a, b);
+          ls[u] = a + b;
+        }
       }
       l_run = fmaf(l_run, alpha, (ls[0] + ls[1]) + (ls[2] + ls[3]));
       m_run = m_new;
@@ -271,12 +310,10 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         if (!ok) break;
         tc_fence_after();
       }
+      // P(j) into TMEM: this thread's row, two bf16 per column, 64 columns
 #pragma unroll
-      for (int c16 = 0; c16 < ATT_BN / 8; ++c16) {          // 16-byte chunks of the 256-byte P row
-        uint8_t* atom_row = p_row + (c16 / 8) * ATOM_BYTES;
-        *reinterpret_cast<uint4*>(atom_row + (((c16 & 7) ^ swz) << 4)) =
-            make_uint4(pk[4 * c16], pk[4 * c16 + 1], pk[4 * c16 + 2], pk[4 * c16 + 3]);
-      }
+      for (int ch = 0; ch < ATT_BN / 64; ++ch)
+        tmem_st32(tmem_p + lane_sel + ch * 32, *reinterpret_cast<const uint32_t(*)[32]>(&pk[ch * 32]));
       // rescale O where the max moved (rows that kept their max multiply by exactly 1)
       if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
 #pragma unroll 1
@@ -288,9 +325,8 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           for (int t = 0; t < 32; ++t) o[t] = __float_as_uint(__uint_as_float(o[t]) * alpha);
           tmem_st32(tmem_o + lane_sel + ch * 32, o);
         }
-        tmem_st_wait();
       }
-      fence_proxy_async_smem();
+      tmem_st_wait();
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(p_full);

@@ -72,6 +72,9 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
         : "r"(smem_u32(bar)), "r"(parity)
         : "memory");
     if (ok) return true;
+#ifdef XEMA_DBG_POLL_SLEEP
+    __nanosleep(XEMA_DBG_POLL_SLEEP);
+#endif
     if ((++polls & 0xFF) == 0) {
       if (*abort_flag) return false;
       if (clock64() - t0 > kWaitLimitCycles) {
@@ -166,6 +169,19 @@ __device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// D[tmem] (+)= A[tmem] * B[smem].  A: lane = row, 16-bit elements packed two per 32-bit column
+// along K (K = 16 elements = 8 columns per instruction), always K-major.
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                       uint32_t accumulate) {
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "setp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n"
+      "}\n"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
 // Makes `bar` complete one arrival once all MMAs issued so far by this thread are done.
 __device__ __forceinline__ void mma_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
@@ -214,6 +230,50 @@ __device__ __forceinline__ float ex2_approx(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+// ---- packed fp32x2 arithmetic (two floats in one 64-bit register pair) ---------------------
+__device__ __forceinline__ uint64_t pack_f32x2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack_f32x2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+// 2^x for two values on the FMA pipe instead of the MUFU: round-to-nearest split x = n + r with
+// |r| <= 1/2 through the 1.5 * 2^23 trick, a cubic for 2^r (relative error 7.5e-5, far below the
+// bf16 rounding of the probabilities it feeds), then n added into the exponent field.
+// Valid for x <= 126; inputs below -125 are clamped (2^-125 stands in for zero).
+__device__ __forceinline__ uint64_t exp2_poly_f32x2(uint64_t x2) {
+  float x0, x1;
+  unpack_f32x2(x2, x0, x1);
+  x2 = pack_f32x2(fmaxf(x0, -125.f), fmaxf(x1, -125.f));
+  const uint64_t magic = pack_f32x2(12582912.f, 12582912.f);
+  const uint64_t neg_magic = pack_f32x2(-12582912.f, -12582912.f);
+  const uint64_t neg_one = pack_f32x2(-1.f, -1.f);
+  const uint64_t t2 = add_f32x2(x2, magic);                 // integer part lands in the low mantissa bits
+  const uint64_t n2 = add_f32x2(t2, neg_magic);             // nearest integer as a float
+  const uint64_t r2 = fma_f32x2(n2, neg_one, x2);           // r = x - n
+  uint64_t p2 = fma_f32x2(pack_f32x2(0.0551716685f, 0.0551716685f), r2, pack_f32x2(0.242611125f, 0.242611125f));
+  p2 = fma_f32x2(p2, r2, pack_f32x2(0.693260968f, 0.693260968f));
+  p2 = fma_f32x2(p2, r2, pack_f32x2(0.999928057f, 0.999928057f));
+  float t0, t1, p0, p1;
+  unpack_f32x2(t2, t0, t1);
+  unpack_f32x2(p2, p0, p1);
+  const float e0 = __uint_as_float(__float_as_uint(p0) + (__float_as_uint(t0) << 23));
+  const float e1 = __uint_as_float(__float_as_uint(p1) + (__float_as_uint(t1) << 23));
+  return pack_f32x2(e0, e1);
+}
+
 // max of three values in one instruction
 __device__ __forceinline__ float max3(float a, float b, float c) {
   float d;
