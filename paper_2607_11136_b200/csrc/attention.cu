@@ -1,21 +1,23 @@
 // Non-causal flash-style attention on tcgen05: o = softmax(q k^T / sqrt(dh)) v over all keys.
 //
-// One CTA owns one (batch, head, 128-query-row tile) and streams the keys in blocks of 128;
-// its workspace (shared memory and TMEM) depends on the query tile only, never on the number
-// of keys.  192 threads:
-//   warp 0    TMA producer: Q tile once, then K and V tiles through two-stage rings
-//   warp 1    owns TMEM; one thread issues S = Q K^T (TMEM, 128 fp32 columns) and
-//             O += P V (TMEM, dh fp32 columns)
-//   warps 2-5 softmax: thread = query row.  Read S from TMEM, running max / sum in the exp2
-//             domain, write P (bf16, two per column) back into TMEM where the second MMA reads
-//             it as its A operand (shared memory carries only Q, K and V: its bandwidth, not
-//             the tensor pipe, bounds this kernel), rescale O in TMEM when the running max
-//             moved, and at the end normalise O and store it.  The score row is held in registers, so the
-//             S buffer is handed back right after the load and S(j+1) = Q K(j+1)^T runs while
-//             the exponentials of block j are evaluated.
+// One CTA owns one (batch, head, 128-query-row tile) and streams the keys in blocks of 64; its
+// workspace (shared memory and TMEM) depends on the query tile only, never on the number of
+// keys.  Two CTAs share an SM.  192 threads:
+//   warp 0    TMA producer: Q tile once, then K and V tiles through a ring of stages
+//   warp 1    owns TMEM; one thread issues S(j) = Q K(j)^T into one of two TMEM score buffers
+//             and O += P(j) V(j) with P read from TMEM
+//   warps 2-5 softmax: thread = query row.  Reads its score row from TMEM into registers,
+//             keeps the running max / sum in the exp2 domain, writes P(j) (bf16, two per
+//             column) in place over the score buffer it came from, rescales O in TMEM when the
+//             running max moved, and at the end normalises O and stores it.
+// Pipeline: the issuing thread's tcgen05 operations execute in order, so after P(j) is ready
+// it queues PV(j) and then S(j+2) into the buffer PV(j) frees; the softmax warps therefore
+// find S(j+1) waiting and depend on the tensor pipe again only in the rare iterations in which
+// a row's running max moved (O must then be at rest).  Shared memory carries only Q, K, V.
+//
 // Every decision is taken per row (the running max only moves when it grows by more than 2^8
 // in the exp2 domain; multiplying the other rows by exactly 1 changes nothing), keys are
-// always visited from key 0 in blocks of 128, and nothing is split or reduced across CTAs, so
+// always visited from key 0 in blocks of 64, and nothing is split or reduced across CTAs, so
 // a query row's output bits do not depend on how the query rows are chunked or tiled.
 #include <algorithm>
 
@@ -26,12 +28,13 @@ namespace xema {
 using namespace sm100;
 
 constexpr int ATT_BM = 128;      // query rows per CTA
-constexpr int ATT_BN = 128;      // keys per block
+constexpr int ATT_BN = 64;       // keys per block
 constexpr int ATT_THREADS = 192;
-constexpr int ATOM_BYTES = 128 * 128;   // 128 rows x 64 bf16, one swizzled column block
+constexpr int Q_ATOM_BYTES = ATT_BM * 128;    // 128 rows x 64 bf16, one swizzled column block
+constexpr int KV_ATOM_BYTES = ATT_BN * 128;   // 64 keys x 64 bf16
 // share of the exponentials evaluated as a polynomial on the FMA pipe instead of the MUFU
 #ifndef XEMA_ATT_POLY_NUM
-#define XEMA_ATT_POLY_NUM 1
+#define XEMA_ATT_POLY_NUM 0
 #endif
 #ifndef XEMA_ATT_POLY_DEN
 #define XEMA_ATT_POLY_DEN 4
@@ -40,23 +43,19 @@ constexpr int POLY_NUM = XEMA_ATT_POLY_NUM, POLY_DEN = XEMA_ATT_POLY_DEN;
 
 template <int DH>
 struct AttnCfg {
-  static constexpr int ATOMS = DH / 64;                      // 64-wide column blocks per tile
-  static constexpr int TILE_BYTES = ATOMS * ATOM_BYTES;      // Q, K or V tile
-  static constexpr int KV_STAGES = (DH == 64) ? 3 : 2;
+  static constexpr int ATOMS = DH / 64;                        // 64-wide column blocks per tile
+  static constexpr int Q_BYTES = ATOMS * Q_ATOM_BYTES;
+  static constexpr int KV_BYTES = ATOMS * KV_ATOM_BYTES;       // one K or V tile
+  static constexpr int KV_STAGES = (DH == 64) ? 4 : 2;
   static constexpr int OFF_Q = 0;
-  static constexpr int OFF_K = OFF_Q + TILE_BYTES;
-  static constexpr int OFF_V = OFF_K + KV_STAGES * TILE_BYTES;
-  static constexpr int OFF_BAR = OFF_V + KV_STAGES * TILE_BYTES;
+  static constexpr int OFF_K = OFF_Q + Q_BYTES;
+  static constexpr int OFF_V = OFF_K + KV_STAGES * KV_BYTES;
+  static constexpr int OFF_BAR = OFF_V + KV_STAGES * KV_BYTES;
   static constexpr int SMEM_BYTES = OFF_BAR + 256;
-  // TMEM columns: S fp32 [0,128); P bf16, two per column [128,192); O fp32 [192, 192+DH)
-  static constexpr int TMEM_P = 128;
-  static constexpr int TMEM_O = 192;
-  static constexpr int TMEM_COLS = (DH == 64) ? 256 : 512;
-#ifdef XEMA_DBG_ONE_CTA
-  static constexpr int MIN_CTAS = 1;
-#else
-  static constexpr int MIN_CTAS = (DH == 64) ? 2 : 1;
-#endif
+  // TMEM columns: two score buffers S0 [0,64), S1 [64,128) (P(j) overwrites the first 32
+  // columns of the buffer S(j) came from); O fp32 [128, 128+DH)
+  static constexpr int TMEM_O = 128;
+  static constexpr int TMEM_COLS = 256;
 };
 
 struct AttnParams {
@@ -69,22 +68,22 @@ struct AttnParams {
 };
 
 template <int DH>
-__global__ void __launch_bounds__(ATT_THREADS, AttnCfg<DH>::MIN_CTAS)
+__global__ void __launch_bounds__(ATT_THREADS, 2)
 attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                  const __grid_constant__ CUtensorMap map_v, const AttnParams p) {
   using Cfg = AttnCfg<DH>;
+  constexpr int STAGES = Cfg::KV_STAGES;
   extern __shared__ __align__(1024) uint8_t smem[];
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + Cfg::OFF_BAR);
   uint64_t* q_full = bars + 0;
-  uint64_t* k_full = bars + 1;    // [KV_STAGES <= 3]
-  uint64_t* k_empty = bars + 4;
-  uint64_t* v_full = bars + 7;
-  uint64_t* v_empty = bars + 10;
-  uint64_t* s_full = bars + 13;
-  uint64_t* p_full = bars + 14;
-  uint64_t* pv_done = bars + 15;
-  uint64_t* s_free = bars + 16;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 17);
+  uint64_t* k_full = bars + 1;    // [STAGES <= 4]
+  uint64_t* k_empty = bars + 5;
+  uint64_t* v_full = bars + 9;
+  uint64_t* v_empty = bars + 13;
+  uint64_t* s_full = bars + 17;   // [2] one per score buffer
+  uint64_t* p_full = bars + 19;   // [2]
+  uint64_t* pv_done = bars + 21;  // [2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 23);
   volatile uint32_t* abort_flag = tmem_slot + 1;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -99,16 +98,17 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 
   if (threadIdx.x == 0) {
     mbar_init(q_full, 1);
-    for (int s = 0; s < Cfg::KV_STAGES; ++s) {
+    for (int s = 0; s < STAGES; ++s) {
       mbar_init(&k_full[s], 1);
       mbar_init(&k_empty[s], 1);
       mbar_init(&v_full[s], 1);
       mbar_init(&v_empty[s], 1);
     }
-    mbar_init(s_full, 1);
-    mbar_init(p_full, 4);
-    mbar_init(s_free, 4);
-    mbar_init(pv_done, 1);
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(&s_full[s], 1);
+      mbar_init(&p_full[s], 4);
+      mbar_init(&pv_done[s], 1);
+    }
     *abort_flag = 0;
     fence_mbar_init();
     prefetch_tmap(&map_q);
@@ -123,101 +123,131 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const uint32_t tmem_s = tmem_base;
-  const uint32_t tmem_p = tmem_base + Cfg::TMEM_P;
   const uint32_t tmem_o = tmem_base + Cfg::TMEM_O;
 
   if (warp == 0) {
     // ---------------- TMA producer ----------------
     if (lane == 0) {
       bool ok = true;
-      mbar_expect_tx(q_full, Cfg::TILE_BYTES);
+      mbar_expect_tx(q_full, Cfg::Q_BYTES);
 #pragma unroll
       for (int a = 0; a < Cfg::ATOMS; ++a)
-        tma_load_3d(smem + Cfg::OFF_Q + a * ATOM_BYTES, &map_q, q_full, h * DH + a * 64, qt * ATT_BM, b);
+        tma_load_3d(smem + Cfg::OFF_Q + a * Q_ATOM_BYTES, &map_q, q_full, h * DH + a * 64, qt * ATT_BM, b);
       int k_issued = 0, v_issued = 0;
+      int st = 0;
+      uint32_t ph = 0;
       for (int j = 0; j < n_kv; ++j) {
-        const int st = j % Cfg::KV_STAGES;
-        const uint32_t ph = (uint32_t)(j / Cfg::KV_STAGES) & 1u;
         if (!(ok = mbar_wait(&k_empty[st], ph ^ 1, abort_flag))) break;
-        mbar_expect_tx(&k_full[st], Cfg::TILE_BYTES);
+        mbar_expect_tx(&k_full[st], Cfg::KV_BYTES);
 #pragma unroll
         for (int a = 0; a < Cfg::ATOMS; ++a)
-          tma_load_3d(smem + Cfg::OFF_K + st * Cfg::TILE_BYTES + a * ATOM_BYTES, &map_k, &k_full[st],
+          tma_load_3d(smem + Cfg::OFF_K + st * Cfg::KV_BYTES + a * KV_ATOM_BYTES, &map_k, &k_full[st],
                       h * DH + a * 64, j * ATT_BN, b);
         k_issued = j + 1;
         if (!(ok = mbar_wait(&v_empty[st], ph ^ 1, abort_flag))) break;
-        mbar_expect_tx(&v_full[st], Cfg::TILE_BYTES);
+        mbar_expect_tx(&v_full[st], Cfg::KV_BYTES);
 #pragma unroll
         for (int a = 0; a < Cfg::ATOMS; ++a)
-          tma_load_3d(smem + Cfg::OFF_V + st * Cfg::TILE_BYTES + a * ATOM_BYTES, &map_v, &v_full[st],
+          tma_load_3d(smem + Cfg::OFF_V + st * Cfg::KV_BYTES + a * KV_ATOM_BYTES, &map_v, &v_full[st],
                       h * DH + a * 64, j * ATT_BN, b);
         v_issued = j + 1;
+        if (++st == STAGES) { st = 0; ph ^= 1; }
       }
       if (!ok) {
         // gave up: let the copies already issued land before the CTA leaves (the latest
         // fill of each stage; older fills were consumed before their stage was reused)
         volatile uint32_t dummy = 0;
         mbar_wait(q_full, 0, &dummy);
-        for (int j = max(0, k_issued - Cfg::KV_STAGES); j < k_issued; ++j) {
+        for (int j = max(0, k_issued - STAGES); j < k_issued; ++j) {
           dummy = 0;
-          mbar_wait(&k_full[j % Cfg::KV_STAGES], (uint32_t)(j / Cfg::KV_STAGES) & 1u, &dummy);
+          mbar_wait(&k_full[j % STAGES], (uint32_t)(j / STAGES) & 1u, &dummy);
         }
-        for (int j = max(0, v_issued - Cfg::KV_STAGES); j < v_issued; ++j) {
+        for (int j = max(0, v_issued - STAGES); j < v_issued; ++j) {
           dummy = 0;
-          mbar_wait(&v_full[j % Cfg::KV_STAGES], (uint32_t)(j / Cfg::KV_STAGES) & 1u, &dummy);
+          mbar_wait(&v_full[j % STAGES], (uint32_t)(j / STAGES) & 1u, &dummy);
         }
       }
     }
   } else if (warp == 1) {
     // ---------------- MMA issuer ----------------
-    if (lane == 0) {
-      constexpr uint32_t idesc_s = idesc_bf16_f32(ATT_BM, ATT_BN, false, false);   // S = Q K^T
-      constexpr uint32_t idesc_o = idesc_bf16_f32(ATT_BM, DH, false, true);        // O = P V, V is N-major
-      const uint32_t q_addr = smem_u32(smem + Cfg::OFF_Q);
-      auto issue_s = [&](int j) -> bool {
-        const int st = j % Cfg::KV_STAGES;
-        const uint32_t ph = (uint32_t)(j / Cfg::KV_STAGES) & 1u;
-        if (!mbar_wait(&k_full[st], ph, abort_flag)) return false;
-        tc_fence_after();
-        const uint32_t k_addr = smem_u32(smem + Cfg::OFF_K + st * Cfg::TILE_BYTES);
+    // The whole warp runs this loop converged and one elected lane issues: descriptors and
+    // barrier addresses then stay warp-uniform values (a lone divergent thread would have to
+    // move every operand into the uniform datapath one by one, and its dependent instruction
+    // stream, not the tensor pipe, would bound the kernel).
+    constexpr uint32_t idesc_s = idesc_bf16_f32(ATT_BM, ATT_BN, false, false);   // S = Q K^T
+    constexpr uint32_t idesc_o = idesc_bf16_f32(ATT_BM, DH, false, true);        // O = P V, V is N-major
+    const uint64_t q_desc = smem_desc_sw128(smem_u32(smem + Cfg::OFF_Q), 16, 1024);
+    const uint64_t k_desc0 = smem_desc_sw128(smem_u32(smem + Cfg::OFF_K), 16, 1024);
+    // V tile: rows = keys (the MMA's K), 64 dh per 128-byte row, 16 keys = 2048 bytes; the
+    // second 64-wide dh block (dh = 128) starts one atom further (leading byte offset)
+    const uint64_t v_desc0 = smem_desc_sw128(smem_u32(smem + Cfg::OFF_V), KV_ATOM_BYTES, 1024);
+    int k_st = 0, v_st = 0;
+    uint32_t k_ph = 0, v_ph = 0;
+    auto wait_all = [&](uint64_t* bar, uint32_t parity) -> bool {
+      return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
+    };
+    auto issue_s = [&](int buf) -> bool {
+      if (!wait_all(&k_full[k_st], k_ph)) return false;
+      tc_fence_after();
+      if (elect_one()) {
+        const uint64_t k_desc = k_desc0 + (uint64_t)(k_st * (Cfg::KV_BYTES >> 4));
+        const uint32_t d = tmem_base + buf * ATT_BN;
 #pragma unroll
-        for (int k = 0; k < DH / 16; ++k) {
-          const uint32_t off = (k / 4) * ATOM_BYTES + (k % 4) * 32;
-          mma_ss(tmem_s, smem_desc_sw128(q_addr + off, 16, 1024), smem_desc_sw128(k_addr + off, 16, 1024), idesc_s,
-                 k != 0);
-        }
-        mma_commit(&k_empty[st]);
-        mma_commit(s_full);
-        return true;
-      };
-      bool ok = mbar_wait(q_full, 0, abort_flag);
-      if (ok) ok = issue_s(0);
-      for (int j = 0; ok && j < n_kv; ++j) {
-        const int st = j % Cfg::KV_STAGES;
-        const uint32_t ph = (uint32_t)(j / Cfg::KV_STAGES) & 1u;
-        // as soon as the softmax warps hold S(j) in registers, S(j+1) may overwrite it
-        if (j + 1 < n_kv) {
-          if (!(ok = mbar_wait(s_free, j & 1, abort_flag))) break;
-          tc_fence_after();
-          if (!(ok = issue_s(j + 1))) break;
-        }
-        // P(j) is in shared memory (and O has been rescaled if the max moved)
-        if (!(ok = mbar_wait(p_full, j & 1, abort_flag))) break;
-        if (!(ok = mbar_wait(&v_full[st], ph, abort_flag))) break;
-        tc_fence_after();
-        const uint32_t v_addr = smem_u32(smem + Cfg::OFF_V + st * Cfg::TILE_BYTES);
-#pragma unroll
-        for (int kk = 0; kk < ATT_BN / 16; ++kk) {
-          // P from TMEM: 16 keys = 8 packed columns per instruction.
-          // V tile: rows = keys (the MMA's K), 64 dh per 128-byte row; 16 keys = 2048 bytes;
-          // the second 64-wide dh block (dh = 128) starts one atom further
-          const uint64_t db = smem_desc_sw128(v_addr + kk * 2048, ATOM_BYTES, 1024);
-          mma_ts(tmem_o, tmem_p + kk * 8, db, idesc_o, (j | kk) != 0);
-        }
-        mma_commit(&v_empty[st]);
-        mma_commit(pv_done);
+        for (int k = 0; k < DH / 16; ++k)
+          mma_ss(d, q_desc + (uint64_t)(((k / 4) * Q_ATOM_BYTES + (k % 4) * 32) >> 4),
+                 k_desc + (uint64_t)(((k / 4) * KV_ATOM_BYTES + (k % 4) * 32) >> 4), idesc_s, k != 0);
+        mma_commit(&k_empty[k_st]);
+        mma_commit(&s_full[buf]);
       }
+      __syncwarp();
+      if (++k_st == STAGES) { k_st = 0; k_ph ^= 1; }
+      return true;
+    };
+    bool ok = wait_all(q_full, 0);
+    if (ok) ok = issue_s(0);
+    if (ok && n_kv > 1) ok = issue_s(1);
+    for (int j = 0; ok && j < n_kv; ++j) {
+      const int buf = j & 1;
+      const uint32_t par = (uint32_t)(j >> 1) & 1u;
+      const bool more = j + 2 < n_kv;
+      // K(j+2) and V(j) were loaded stages ahead: check them while P(j) is still being made,
+      // so that nothing stands between P(j) becoming ready and the two products being queued
+      // (only with a deep ring: with two stages K(j+2) is requested too late for that)
+      constexpr bool kEarlyK = STAGES >= 4;
+      if (kEarlyK && more && !(ok = wait_all(&k_full[k_st], k_ph))) break;
+      if (!(ok = wait_all(&v_full[v_st], v_ph))) break;
+      // P(j) sits in TMEM over S(j) (and O has been rescaled if a running max moved)
+      if (!(ok = wait_all(&p_full[buf], par))) break;
+      tc_fence_after();
+      if (elect_one()) {
+        const uint64_t v_desc = v_desc0 + (uint64_t)(v_st * (Cfg::KV_BYTES >> 4));
+        const uint32_t sp_tmem = tmem_base + buf * ATT_BN;
+#pragma unroll
+        for (int kk = 0; kk < ATT_BN / 16; ++kk)             // 16 keys = 8 packed P columns
+          mma_ts(tmem_o, sp_tmem + kk * 8, v_desc + (uint64_t)(kk * (2048 >> 4)), idesc_o, (j | kk) != 0);
+        mma_commit(&v_empty[v_st]);
+        mma_commit(&pv_done[buf]);
+      }
+      if (!kEarlyK && more) {
+        if (!(ok = wait_all(&k_full[k_st], k_ph))) break;
+        tc_fence_after();
+      }
+      if (elect_one()) {
+        const uint32_t sp_tmem = tmem_base + buf * ATT_BN;
+        // S(j+2) reuses the buffer; it is queued behind PV(j), which reads P(j) from it
+        if (more) {
+          const uint64_t k_desc = k_desc0 + (uint64_t)(k_st * (Cfg::KV_BYTES >> 4));
+#pragma unroll
+          for (int k = 0; k < DH / 16; ++k)
+            mma_ss(sp_tmem, q_desc + (uint64_t)(((k / 4) * Q_ATOM_BYTES + (k % 4) * 32) >> 4),
+                   k_desc + (uint64_t)(((k / 4) * KV_ATOM_BYTES + (k % 4) * 32) >> 4), idesc_s, k != 0);
+          mma_commit(&k_empty[k_st]);
+          mma_commit(&s_full[buf]);
+        }
+      }
+      __syncwarp();
+      if (++v_st == STAGES) { v_st = 0; v_ph ^= 1; }
+      if (more && ++k_st == STAGES) { k_st = 0; k_ph ^= 1; }
     }
   } else {
     // ---------------- softmax / correction / epilogue ----------------
@@ -226,20 +256,24 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     const uint32_t lane_sel = (uint32_t)(quad * 32) << 16;
     float m_run = -INFINITY, l_run = 0.f;
     bool ok = true;
-    for (int j = 0; j < n_kv; ++j) {
-      ok = mbar_wait(s_full, j & 1, abort_flag);
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) break;
+    // The score row of block j+1 is requested from TMEM as soon as the registers of block j
+    // are free (its exponentials are done), so the load and the barrier check overlap the
+    // store of P(j); s[] always holds the block that is being worked on.
+    float s[ATT_BN];
+    ok = __all_sync(0xffffffffu, mbar_wait(&s_full[0], 0, abort_flag));
+    if (ok) {
       tc_fence_after();
-      // the whole score row of this thread into registers, then hand the TMEM buffer back
-      float s[ATT_BN];
 #pragma unroll
       for (int ch = 0; ch < ATT_BN / 32; ++ch)
-        tmem_ld32(tmem_s + lane_sel + ch * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[ch * 32]));
+        tmem_ld32(tmem_base + lane_sel + ch * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[ch * 32]));
+    }
+    for (int j = 0; ok && j < n_kv; ++j) {
+      const int buf = j & 1;
+      const uint32_t s_tmem = tmem_base + lane_sel + buf * ATT_BN;
+      const uint32_t next_par = (uint32_t)((j + 1) >> 1) & 1u;
       tmem_ld_wait();
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(s_free);
+      // look at S(j+1)'s barrier now; the answer is needed only after the exponentials
+      const bool next_ready = (j + 1 < n_kv) && mbar_test(&s_full[buf ^ 1], next_par);
       // keys past the end exist only in the last block
       const int valid = p.keys - j * ATT_BN;
       if (valid < ATT_BN) {
@@ -247,17 +281,16 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         for (int t = 0; t < ATT_BN; ++t)
           if (t >= valid) s[t] = -INFINITY;
       }
-      // row max: independent partial maxima, three-input max
-      float mx[8];
+      // row max: independent chains of three-input max
+      float mx[4];
 #pragma unroll
-      for (int u = 0; u < 8; ++u) mx[u] = max3(s[16 * u], s[16 * u + 1], s[16 * u + 2]);
-#pragma unroll
-      for (int u = 0; u < 8; ++u) {
+      for (int u = 0; u < 4; ++u) {
+        mx[u] = max3(s[16 * u], s[16 * u + 1], s[16 * u + 2]);
 #pragma unroll
         for (int t = 3; t < 15; t += 2) mx[u] = max3(mx[u], s[16 * u + t], s[16 * u + t + 1]);
         mx[u] = fmaxf(mx[u], s[16 * u + 15]);
       }
-      const float m_blk = fmaxf(max3(mx[0], mx[1], mx[2]), max3(max3(mx[3], mx[4], mx[5]), mx[6], mx[7]));
+      const float m_blk = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
       // the running max moves only when it grows by more than 2^8 (exp2 domain); per row
       float m_new = m_run;
       if (j == 0 || (m_blk - m_run) * p.scale_log2 > 8.f) m_new = m_blk;
@@ -280,13 +313,8 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           unpack_f32x2(e2, e0, e1);
         } else {
           unpack_f32x2(e2, e0, e1);
-#ifdef XEMA_DBG_NOEXP
-          e0 = e0 * 0.001f + 1.f;
-          e1 = e1 * 0.001f + 1.f;
-#else
           e0 = ex2_approx(e0);
           e1 = ex2_approx(e1);
-#endif
           e2 = pack_f32x2(e0, e1);
         }
         ls2[pair & 3] = add_f32x2(ls2[pair & 3], e2);
@@ -294,28 +322,22 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       }
       float ls[4];
       {
-        float a, b;
+        float a0, a1;
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-          unpack_f32x2(ls2[u], a, b);
-          ls[u] = a + b;
+          unpack_f32x2(ls2[u], a0, a1);
+          ls[u] = a0 + a1;
         }
       }
       l_run = fmaf(l_run, alpha, (ls[0] + ls[1]) + (ls[2] + ls[3]));
       m_run = m_new;
-      // P(j) overwrites the buffer PV(j-1) reads, and O must be at rest before it is rescaled
-      if (j > 0) {
-        ok = mbar_wait(pv_done, (j - 1) & 1, abort_flag);
+      // rescale O where the max moved (rows that kept their max multiply by exactly 1); only
+      // then must PV(j-1) have finished
+      if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+        ok = mbar_wait(&pv_done[(j - 1) & 1], (uint32_t)((j - 1) >> 1) & 1u, abort_flag);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after();
-      }
-      // P(j) into TMEM: this thread's row, two bf16 per column, 64 columns
-#pragma unroll
-      for (int ch = 0; ch < ATT_BN / 64; ++ch)
-        tmem_st32(tmem_p + lane_sel + ch * 32, *reinterpret_cast<const uint32_t(*)[32]>(&pk[ch * 32]));
-      // rescale O where the max moved (rows that kept their max multiply by exactly 1)
-      if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
 #pragma unroll 1
         for (int ch = 0; ch < DH / 32; ++ch) {
           uint32_t o[32];
@@ -326,13 +348,26 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           tmem_st32(tmem_o + lane_sel + ch * 32, o);
         }
       }
+      // P(j) in place over this thread's score row: two bf16 per column, 32 columns
+      tmem_st32(s_tmem, pk);
+      if (j + 1 < n_kv) {
+        if (!__all_sync(0xffffffffu, next_ready)) {
+          ok = __all_sync(0xffffffffu, mbar_wait(&s_full[buf ^ 1], next_par, abort_flag));
+          if (!ok) break;
+        }
+        tc_fence_after();
+#pragma unroll
+        for (int ch = 0; ch < ATT_BN / 32; ++ch)
+          tmem_ld32(tmem_base + lane_sel + (buf ^ 1) * ATT_BN + ch * 32,
+                    *reinterpret_cast<uint32_t(*)[32]>(&s[ch * 32]));
+      }
       tmem_st_wait();
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(p_full);
+      if (lane == 0) mbar_arrive(&p_full[buf]);
     }
     if (ok) {
-      ok = mbar_wait(pv_done, (n_kv - 1) & 1, abort_flag);
+      ok = mbar_wait(&pv_done[(n_kv - 1) & 1], (uint32_t)((n_kv - 1) >> 1) & 1u, abort_flag);
       ok = __all_sync(0xffffffffu, ok);
     }
     if (ok) {

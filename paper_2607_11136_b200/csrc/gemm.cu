@@ -210,6 +210,11 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     // ---------------- MMA issuer ----------------
     if (lane == 0) {
       constexpr uint32_t idesc = idesc_bf16_f32(BM, BN, false, false);
+      // The issuing thread is a lone dependent instruction stream, so its loop is kept short:
+      // descriptors are built once and advanced by adding constants (the start-address field
+      // counts 16-byte units and never carries out of its 14 bits inside shared memory).
+      const uint64_t a_desc0 = smem_desc_sw128(smem_u32(smem), 16, 1024);
+      const uint64_t b_desc0 = smem_desc_sw128(smem_u32(smem + A_TILE_BYTES), 16, 1024);
       int stage = 0;
       uint32_t phase = 0;
       int acc = 0;
@@ -219,18 +224,19 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         if (!(ok = mbar_wait(&tmem_empty[acc], acc_phase ^ 1, abort_flag))) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * BN;
+        uint32_t accumulate = 0;
+#pragma unroll 1
         for (int kb = 0; kb < k_blocks; ++kb) {
           if (!(ok = mbar_wait(&full[stage], phase, abort_flag))) break;
           tc_fence_after();
-          const uint32_t a_addr = smem_u32(smem + stage * Cfg::STAGE_BYTES);
-          const uint32_t b_addr = a_addr + A_TILE_BYTES;
-#pragma unroll
-          for (int k = 0; k < BK / 16; ++k) {
-            const uint64_t da = smem_desc_sw128(a_addr + k * 32, 16, 1024);
-            const uint64_t db = smem_desc_sw128(b_addr + k * 32, 16, 1024);
-            mma_ss(d_tmem, da, db, idesc, (kb | k) != 0);
-          }
+          const uint64_t soff = (uint64_t)(stage * (Cfg::STAGE_BYTES >> 4));
+          const uint64_t da = a_desc0 + soff, db = b_desc0 + soff;
+          mma_ss(d_tmem, da, db, idesc, accumulate);
+          mma_ss(d_tmem, da + 2, db + 2, idesc, 1);
+          mma_ss(d_tmem, da + 4, db + 4, idesc, 1);
+          mma_ss(d_tmem, da + 6, db + 6, idesc, 1);
           mma_commit(&empty[stage]);
+          accumulate = 1;
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
         if (!ok) break;

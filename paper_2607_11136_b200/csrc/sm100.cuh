@@ -47,8 +47,8 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
 }
 // Bounded wait.  Returns false when the limit ran out (the caller then abandons its loop);
 // `abort_flag` (shared memory) lets the CTA's other roles stop early once one of them gave up.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag) {
-  uint32_t ok = 0;
+__device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
   asm volatile(
       "{\n"
       ".reg .pred p;\n"
@@ -58,24 +58,14 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
       : "=r"(ok)
       : "r"(smem_u32(bar)), "r"(parity)
       : "memory");
-  if (ok) return true;
+  return ok != 0;
+}
+static __device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag) {
   const long long t0 = clock64();
   uint32_t polls = 0;
   while (true) {
-    asm volatile(
-        "{\n"
-        ".reg .pred p;\n"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-        "selp.u32 %0, 1, 0, p;\n"
-        "}\n"
-        : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
-    if (ok) return true;
-#ifdef XEMA_DBG_POLL_SLEEP
-    __nanosleep(XEMA_DBG_POLL_SLEEP);
-#endif
-    if ((++polls & 0xFF) == 0) {
+    if (mbar_test(bar, parity)) return true;
+    if ((++polls & 0x3F) == 0) {
       if (*abort_flag) return false;
       if (clock64() - t0 > kWaitLimitCycles) {
         *abort_flag = 1;
@@ -83,6 +73,13 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
       }
     }
   }
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag) {
+  // fast path: a few plain polls with nothing else in the dependent chain
+#pragma unroll 1
+  for (int i = 0; i < 8; ++i)
+    if (mbar_test(bar, parity)) return true;
+  return mbar_wait_slow(bar, parity, abort_flag);
 }
 
 // ---- fences ----------------------------------------------------------------------------
