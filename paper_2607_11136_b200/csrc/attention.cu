@@ -256,9 +256,8 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     const uint32_t lane_sel = (uint32_t)(quad * 32) << 16;
     float m_run = -INFINITY, l_run = 0.f;
     bool ok = true;
-    // The score row of block j+1 is requested from TMEM as soon as the registers of block j
-    // are free (its exponentials are done), so the load and the barrier check overlap the
-    // store of P(j); s[] always holds the block that is being worked on.
+    // The score row of block j+1 is requested from TMEM at the end of iteration j, right after
+    // P(j) has been handed over; s[] always holds the block that is being worked on.
     float s[ATT_BN];
     ok = __all_sync(0xffffffffu, mbar_wait(&s_full[0], 0, abort_flag));
     if (ok) {
@@ -272,8 +271,6 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       const uint32_t s_tmem = tmem_base + lane_sel + buf * ATT_BN;
       const uint32_t next_par = (uint32_t)((j + 1) >> 1) & 1u;
       tmem_ld_wait();
-      // look at S(j+1)'s barrier now; the answer is needed only after the exponentials
-      const bool next_ready = (j + 1 < n_kv) && mbar_test(&s_full[buf ^ 1], next_par);
       // keys past the end exist only in the last block
       const int valid = p.keys - j * ATT_BN;
       if (valid < ATT_BN) {
@@ -350,21 +347,20 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       }
       // P(j) in place over this thread's score row: two bf16 per column, 32 columns
       tmem_st32(s_tmem, pk);
+      tmem_st_wait();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&p_full[buf]);
+      // request the next score row (S(j+1) was queued while this block was being worked on)
       if (j + 1 < n_kv) {
-        if (!__all_sync(0xffffffffu, next_ready)) {
-          ok = __all_sync(0xffffffffu, mbar_wait(&s_full[buf ^ 1], next_par, abort_flag));
-          if (!ok) break;
-        }
+        ok = __all_sync(0xffffffffu, mbar_wait(&s_full[buf ^ 1], next_par, abort_flag));
+        if (!ok) break;
         tc_fence_after();
 #pragma unroll
         for (int ch = 0; ch < ATT_BN / 32; ++ch)
           tmem_ld32(tmem_base + lane_sel + (buf ^ 1) * ATT_BN + ch * 32,
                     *reinterpret_cast<uint32_t(*)[32]>(&s[ch * 32]));
       }
-      tmem_st_wait();
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&p_full[buf]);
     }
     if (ok) {
       ok = mbar_wait(&pv_done[(n_kv - 1) & 1], (uint32_t)((n_kv - 1) >> 1) & 1u, abort_flag);
