@@ -430,7 +430,7 @@ static int launch_attention_t(const AttnLaunch& a, cudaStream_t stream) {
 
 int launch_attention(const AttnLaunch& a, cudaStream_t stream) {
   if (a.rows == 0 || a.batch == 0) return XEMA_OK;
-  if (a.head_dim == 64) return launch_attention_t<64>(a, stream);
+  if (a.head_dim == 64) return launch_attention_dh64(a, stream);
   if (a.head_dim == 128) return launch_attention_t<128>(a, stream);
   return XEMA_EINVAL;
 }

@@ -57,5 +57,6 @@ struct AttnLaunch {
 int attn_prepare(AttnLaunch* a, const void* q, long long ldq, long long q_batch_rows, const void* k, const void* v,
                  long long ldkv, long long kv_batch_rows);
 int launch_attention(const AttnLaunch& a, cudaStream_t stream);
+int launch_attention_dh64(const AttnLaunch& a, cudaStream_t stream);   // two-tile kernel for head_dim 64
 
 }  // namespace xema
