@@ -60,6 +60,10 @@ __device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+// Upper bound, in nanoseconds, for which one try_wait of the slow path may park the thread.
+#ifndef XEMA_WAIT_HINT_NS
+#define XEMA_WAIT_HINT_NS 1000u
+#endif
 // Non-blocking look at a barrier phase (try_wait may park the thread for a while when the phase
 // is still open; test_wait returns at once).
 __device__ __forceinline__ bool mbar_peek(uint64_t* bar, uint32_t parity) {
@@ -79,7 +83,17 @@ static __device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parit
   const long long t0 = clock64();
   uint32_t polls = 0;
   while (true) {
-    if (mbar_test(bar, parity)) return true;
+    uint32_t ok;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity), "r"(XEMA_WAIT_HINT_NS)
+        : "memory");
+    if (ok) return true;
     if ((++polls & 0x3F) == 0) {
       if (*abort_flag) return false;
       if (clock64() - t0 > kWaitLimitCycles) {
