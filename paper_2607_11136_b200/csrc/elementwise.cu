@@ -1,6 +1,8 @@
 // HBM-bound kernels of the block: adaLN modulation GEMV, LayerNorm + modulate, and
 // per-head RMSNorm + RoPE.  128-bit coalesced accesses, one warp per token row, warp-shuffle
 // reductions, fp32 arithmetic on bf16 storage.
+#include <algorithm>
+
 #include "kernels.h"
 #include "sm100.cuh"
 
@@ -193,11 +195,102 @@ ln_modulate_kernel(const void* __restrict__ in, long long in_batch_rows, __nv_bf
   }
 }
 
+// Wide rows (D a multiple of 1024): one 128-thread block per row, 8 consecutive features per
+// thread and step.  A thread then holds only D/128 values, so many more warps are resident and
+// enough loads are in flight to cover the HBM latency; the two reductions go through shared
+// memory.  Same arithmetic as above (mean, then centred sum of squares).
+constexpr int kLnRowThreads = 128;
+
+__device__ __forceinline__ float block_sum_128(float v, float* red, int phase) {
+  v = warp_sum(v);
+  float* slot = red + phase * 4;
+  if ((threadIdx.x & 31) == 0) slot[threadIdx.x >> 5] = v;
+  __syncthreads();
+  return (slot[0] + slot[1]) + (slot[2] + slot[3]);
+}
+
+template <bool IN_F32, int VPT>
+__global__ void __launch_bounds__(kLnRowThreads)
+ln_modulate_row_kernel(const void* __restrict__ in, long long in_batch_rows, __nv_bfloat16* __restrict__ out,
+                       const float* __restrict__ shift, const float* __restrict__ scale, long long mod_stride,
+                       int batch, int rows, int D, float eps) {
+  __shared__ float red[16];
+  const long long total = (long long)batch * rows;
+  const float inv_d = 1.f / (float)D;
+  int parity = 0;
+  for (long long r = blockIdx.x; r < total; r += gridDim.x, parity ^= 2) {
+    const int b = (int)(r / rows);
+    const int i = (int)(r - (long long)b * rows);
+    const size_t in_elem = ((size_t)b * in_batch_rows + i) * D;
+    const float* sh = shift + (size_t)b * mod_stride;
+    const float* sc = scale + (size_t)b * mod_stride;
+    float x[VPT][8];
+    float s = 0.f;
+#pragma unroll
+    for (int v = 0; v < VPT; ++v) {
+      const int e0 = (v * kLnRowThreads + threadIdx.x) * 8;
+      if constexpr (IN_F32) {
+        const float4* p = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(in) + in_elem + e0);
+        const float4 a = __ldg(p), c = __ldg(p + 1);
+        x[v][0] = a.x; x[v][1] = a.y; x[v][2] = a.z; x[v][3] = a.w;
+        x[v][4] = c.x; x[v][5] = c.y; x[v][6] = c.z; x[v][7] = c.w;
+      } else {
+        const uint4 u = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(in) + in_elem + e0));
+        x[v][0] = bf16_lo(u.x); x[v][1] = bf16_hi(u.x); x[v][2] = bf16_lo(u.y); x[v][3] = bf16_hi(u.y);
+        x[v][4] = bf16_lo(u.z); x[v][5] = bf16_hi(u.z); x[v][6] = bf16_lo(u.w); x[v][7] = bf16_hi(u.w);
+      }
+#pragma unroll
+      for (int t = 0; t < 8; ++t) s += x[v][t];
+    }
+    const float mean = block_sum_128(s, red, parity) * inv_d;
+    float q = 0.f;
+#pragma unroll
+    for (int v = 0; v < VPT; ++v)
+#pragma unroll
+      for (int t = 0; t < 8; ++t) {
+        x[v][t] -= mean;
+        q = fmaf(x[v][t], x[v][t], q);
+      }
+    const float rstd = rsqrtf(block_sum_128(q, red, parity + 1) * inv_d + eps);
+    __nv_bfloat16* dst = out + (size_t)r * D;
+#pragma unroll
+    for (int v = 0; v < VPT; ++v) {
+      const int e0 = (v * kLnRowThreads + threadIdx.x) * 8;
+      const float4 a0 = __ldg(reinterpret_cast<const float4*>(sc + e0)), a1 = __ldg(reinterpret_cast<const float4*>(sc + e0 + 4));
+      const float4 c0 = __ldg(reinterpret_cast<const float4*>(sh + e0)), c1 = __ldg(reinterpret_cast<const float4*>(sh + e0 + 4));
+      const float y0 = fmaf(x[v][0] * rstd, 1.f + a0.x, c0.x), y1 = fmaf(x[v][1] * rstd, 1.f + a0.y, c0.y);
+      const float y2 = fmaf(x[v][2] * rstd, 1.f + a0.z, c0.z), y3 = fmaf(x[v][3] * rstd, 1.f + a0.w, c0.w);
+      const float y4 = fmaf(x[v][4] * rstd, 1.f + a1.x, c1.x), y5 = fmaf(x[v][5] * rstd, 1.f + a1.y, c1.y);
+      const float y6 = fmaf(x[v][6] * rstd, 1.f + a1.z, c1.z), y7 = fmaf(x[v][7] * rstd, 1.f + a1.w, c1.w);
+      *reinterpret_cast<uint4*>(dst + e0) =
+          make_uint4(pack_bf16x2(y0, y1), pack_bf16x2(y2, y3), pack_bf16x2(y4, y5), pack_bf16x2(y6, y7));
+    }
+  }
+}
+
 template <bool IN_F32>
 static int launch_ln_t(const void* in, long long in_batch_rows, void* out, const float* shift, const float* scale,
                        long long mod_stride, int batch, int rows, int D, float eps, cudaStream_t stream) {
   constexpr int EPV = LnIo<IN_F32>::EPV;
   const long long total = (long long)batch * rows;
+  if (D % 1024 == 0 && D / 1024 <= 4) {
+    // 16 resident blocks per SM cover the whole GPU; rows beyond that are taken in a stride loop
+    const unsigned grid = (unsigned)std::min<long long>(total, 148LL * 16);
+    auto* o2 = (__nv_bfloat16*)out;
+#define XEMA_LNROW_CASE(N)                                                                                       \
+  case N:                                                                                                        \
+    ln_modulate_row_kernel<IN_F32, N><<<grid, kLnRowThreads, 0, stream>>>(in, in_batch_rows, o2, shift, scale,   \
+                                                                           mod_stride, batch, rows, D, eps);     \
+    break;
+    switch (D / 1024) {
+      XEMA_LNROW_CASE(1)
+      XEMA_LNROW_CASE(2)
+      XEMA_LNROW_CASE(3)
+      XEMA_LNROW_CASE(4)
+    }
+#undef XEMA_LNROW_CASE
+    return check_launch();
+  }
   const unsigned blocks = (unsigned)((total + kLnWarps - 1) / kLnWarps);
   const int nv = D / (32 * EPV);
   auto* o = (__nv_bfloat16*)out;
