@@ -64,6 +64,10 @@ __device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
 #ifndef XEMA_WAIT_HINT_NS
 #define XEMA_WAIT_HINT_NS 1000u
 #endif
+// Plain polls before a wait moves to the parked slow path.
+#ifndef XEMA_WAIT_FAST_POLLS
+#define XEMA_WAIT_FAST_POLLS 2
+#endif
 // Non-blocking look at a barrier phase (try_wait may park the thread for a while when the phase
 // is still open; test_wait returns at once).
 __device__ __forceinline__ bool mbar_peek(uint64_t* bar, uint32_t parity) {
@@ -106,7 +110,7 @@ static __device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parit
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag) {
   // fast path: a few plain polls with nothing else in the dependent chain
 #pragma unroll 1
-  for (int i = 0; i < 8; ++i)
+  for (int i = 0; i < XEMA_WAIT_FAST_POLLS; ++i)
     if (mbar_test(bar, parity)) return true;
   return mbar_wait_slow(bar, parity, abort_flag);
 }
@@ -240,6 +244,15 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
         "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]),
         "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]),
         "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+// 16 consecutive columns.
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
       : "memory");
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
