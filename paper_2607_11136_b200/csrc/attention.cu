@@ -447,9 +447,11 @@ int attn_prepare(AttnLaunch* a, const void* q, long long ldq, long long q_batch_
   const long long width = (long long)a->heads * a->head_dim;
   int rc = encode_tmap_bf16(&a->map_q, q, width, a->rows > 0 ? a->rows : 1, a->batch, ldq, q_batch_rows, ATT_BM);
   if (rc) return rc;
-  rc = encode_tmap_bf16(&a->map_k, k, width, a->keys, a->batch, ldkv, kv_batch_rows, ATT_BN);
+  // keys per block (= rows of a K/V box): 32 in the head_dim 64 kernel, 64 in the general one
+  const int kv_box = (a->head_dim == 64) ? kAttnDh64KeysPerBlock : ATT_BN;
+  rc = encode_tmap_bf16(&a->map_k, k, width, a->keys, a->batch, ldkv, kv_batch_rows, kv_box);
   if (rc) return rc;
-  return encode_tmap_bf16(&a->map_v, v, width, a->keys, a->batch, ldkv, kv_batch_rows, ATT_BN);
+  return encode_tmap_bf16(&a->map_v, v, width, a->keys, a->batch, ldkv, kv_batch_rows, kv_box);
 }
 
 }  // namespace xema

@@ -26,7 +26,7 @@ using namespace sm100;
 namespace {
 constexpr int BM = 128;          // rows per tile
 constexpr int TILES = 2;
-constexpr int BN = 64;           // keys per block
+constexpr int BN = kAttnDh64KeysPerBlock;   // keys per block (64)
 constexpr int DH = 64;
 constexpr int THREADS = 64 + 128 * TILES;
 constexpr int Q_TILE_BYTES = BM * 128;
@@ -182,23 +182,10 @@ attention_dh64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
       if (!(ok = wait_all(&v_full[v_st], v_ph))) break;
       const uint64_t v_desc = v_desc0 + (uint64_t)(v_st * (KV_TILE_BYTES >> 4));
       const uint64_t k_desc = k_desc0 + (uint64_t)(k_st * (KV_TILE_BYTES >> 4));
-      // Serve the two tiles in the order in which their P(j) becomes ready: look at both
-      // barriers without blocking; after a bounded number of looks fall back to a blocking,
-      // time-limited wait on the first tile still pending.
-      uint32_t pending = (1u << TILES) - 1;
-      uint32_t looks = 0;
-      while (pending) {
-        int t = -1;
 #pragma unroll
-        for (int c = 0; c < TILES; ++c)
-          if (t < 0 && (pending >> c & 1) && __all_sync(0xffffffffu, mbar_peek(&p_full[c], par))) t = c;
-        if (t < 0) {
-          if (++looks < 4096) continue;
-          t = (pending & 1) ? 0 : 1;
-          if (!(ok = wait_all(&p_full[t], par))) break;
-        }
-        pending &= ~(1u << t);
+      for (int t = 0; t < TILES; ++t) {
         // P(j) of this tile sits in TMEM over S(j) (and O was rescaled if a running max moved)
+        if (!(ok = wait_all(&p_full[t], par))) break;
         tc_fence_after();
         if (elect_one()) {
           const uint32_t sp = tmem_base + t * 128;
@@ -206,16 +193,15 @@ attention_dh64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
           for (int kk = 0; kk < BN / 16; ++kk)               // 16 keys = 8 packed P columns
             mma_ts(sp + 64, sp + kk * 8, v_desc + (uint64_t)(kk * (2048 >> 4)), idesc_o, (j | kk) != 0);
           mma_commit(&pv_done[t]);
-          if (pending == 0) mma_commit(&v_empty[v_st]);
+          if (t == TILES - 1) mma_commit(&v_empty[v_st]);
           // S(j+1) goes into the same columns; it is queued behind PV(j), which reads P(j) there
           if (more) {
             issue_s(t, k_desc);
-            if (pending == 0) mma_commit(&k_empty[k_st]);
+            if (t == TILES - 1) mma_commit(&k_empty[k_st]);
           }
         }
         __syncwarp();
       }
-      if (!ok) break;
       if (++v_st == STAGES) { v_st = 0; v_ph ^= 1; }
       if (more && ++k_st == STAGES) { k_st = 0; k_ph ^= 1; }
     }
@@ -228,9 +214,6 @@ attention_dh64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
     const uint32_t o_tmem = s_tmem + 64;
     float m_run = -INFINITY, l_run = 0.f;
     bool ok = true;
-#ifdef XEMA_ATT_SKEW_NS
-    if (tile == 1) __nanosleep(XEMA_ATT_SKEW_NS);
-#endif
     for (int j = 0; j < n_kv; ++j) {
       const uint32_t par = (uint32_t)j & 1u;
       ok = __all_sync(0xffffffffu, mbar_wait(&s_full[tile], par, abort_flag));

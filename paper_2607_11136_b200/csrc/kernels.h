@@ -58,5 +58,6 @@ int attn_prepare(AttnLaunch* a, const void* q, long long ldq, long long q_batch_
                  long long ldkv, long long kv_batch_rows);
 int launch_attention(const AttnLaunch& a, cudaStream_t stream);
 int launch_attention_dh64(const AttnLaunch& a, cudaStream_t stream);   // two-tile kernel for head_dim 64
+constexpr int kAttnDh64KeysPerBlock = 64;                              // rows of its K/V TMA boxes
 
 }  // namespace xema
