@@ -39,7 +39,7 @@ constexpr int OFF_BAR = OFF_V + STAGES * KV_TILE_BYTES;
 constexpr int SMEM_BYTES = OFF_BAR + 256;
 constexpr int TMEM_COLS = 256;   // per tile: S/P [0,64), O [64,128)
 #ifndef XEMA_ATT_POLY_NUM
-#define XEMA_ATT_POLY_NUM 0
+#define XEMA_ATT_POLY_NUM 1
 #endif
 #ifndef XEMA_ATT_POLY_DEN
 #define XEMA_ATT_POLY_DEN 4

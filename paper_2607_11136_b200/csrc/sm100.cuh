@@ -313,6 +313,25 @@ __device__ __forceinline__ uint64_t exp2_poly_f32x2(uint64_t x2) {
   return pack_f32x2(e0, e1);
 }
 
+// Same polynomial for a pair whose inputs are already >= -125; results come back unpacked
+// (the caller packs them to bf16 and adds them to its row sum).
+__device__ __forceinline__ void exp2_poly_pair(uint64_t x2, float& e0, float& e1) {
+  const uint64_t magic = pack_f32x2(12582912.f, 12582912.f);
+  const uint64_t neg_magic = pack_f32x2(-12582912.f, -12582912.f);
+  const uint64_t neg_one = pack_f32x2(-1.f, -1.f);
+  const uint64_t t2 = add_f32x2(x2, magic);
+  const uint64_t n2 = add_f32x2(t2, neg_magic);
+  const uint64_t r2 = fma_f32x2(n2, neg_one, x2);
+  uint64_t p2 = fma_f32x2(pack_f32x2(0.0551716685f, 0.0551716685f), r2, pack_f32x2(0.242611125f, 0.242611125f));
+  p2 = fma_f32x2(p2, r2, pack_f32x2(0.693260968f, 0.693260968f));
+  p2 = fma_f32x2(p2, r2, pack_f32x2(0.999928057f, 0.999928057f));
+  float t0, t1, p0, p1;
+  unpack_f32x2(t2, t0, t1);
+  unpack_f32x2(p2, p0, p1);
+  e0 = __uint_as_float(__float_as_uint(p0) + (__float_as_uint(t0) << 23));
+  e1 = __uint_as_float(__float_as_uint(p1) + (__float_as_uint(t1) << 23));
+}
+
 // max of three values in one instruction
 __device__ __forceinline__ float max3(float a, float b, float c) {
   float d;
