@@ -273,6 +273,18 @@ int xema_op_attention(const void* q, int64_t ldq, int64_t q_batch_rows, const vo
                       void* stream);
 
 /* ---- diagnostics ------------------------------------------------------------------------ */
+/* Every wait inside the kernels (on an mbarrier fed by TMA, by the tensor pipe or by another
+ * warp) is bounded: when the limit runs out the CTA stops, frees its TMEM, stores
+ * XEMA_DEVICE_STATUS_TIMEOUT in the caller's status word and returns; the forward call's work
+ * is then incomplete but the context stays usable.  This self-test launches one small kernel
+ * that waits, with `limit_cycles` (1 .. 4e9 SM clock cycles) as its limit, on a barrier nothing
+ * completes, so the mechanism can be exercised without faulting or hanging a GPU.
+ * status_dev: device, 4 zeroed bytes, receives XEMA_DEVICE_STATUS_TIMEOUT.  waited_cycles_dev:
+ * device int64 or NULL, receives the cycles the wait took. */
+#define XEMA_DEVICE_STATUS_TIMEOUT 0x54310001u
+int xema_selftest_wait_timeout(void* status_dev, int64_t limit_cycles, int64_t* waited_cycles_dev,
+                               void* stream);
+
 const char* xema_strerror(int status);
 /* Last cudaError_t / CUresult seen by this thread's most recent failing call (0 if none). */
 int xema_last_cuda_error(void);

@@ -25,7 +25,7 @@ EXPORTS = (
     "xema_block_forward_static",
     "xema_plan_launch_count", "xema_forward_prefix", "xema_forward_range", "xema_plan_op", "xema_op_mod", "xema_op_ln_modulate",
     "xema_op_rmsnorm_rope", "xema_op_gemm", "xema_op_attention", "xema_strerror",
-    "xema_last_cuda_error", "xema_version",
+    "xema_last_cuda_error", "xema_version", "xema_selftest_wait_timeout",
 )
 
 
@@ -102,6 +102,7 @@ def lib() -> C.CDLL:
             "xema_op_gemm": [P(xema_gemm_args), vp, vp],
             "xema_op_attention": [vp, i64, i64, vp, vp, i64, i64, vp, vp, i32, i32, i32, i32, i32, vp, vp],
             "xema_last_cuda_error": [],
+            "xema_selftest_wait_timeout": [vp, i64, vp, vp],
         }
         for name, args in sig.items():
             fn = getattr(L, name)
@@ -259,6 +260,14 @@ class Plan:
 
     def forward_prefix(self, n_logical_ops: int, stream: int = 0):
         _check(lib().xema_forward_prefix(self._h, n_logical_ops, stream), "xema_forward_prefix")
+
+
+DEVICE_STATUS_TIMEOUT = 0x54310001
+
+
+def xema_selftest_wait_timeout(status: int, limit_cycles: int, waited_cycles: Optional[int] = None, stream: int = 0):
+    _check(lib().xema_selftest_wait_timeout(status, limit_cycles, waited_cycles, stream),
+           "xema_selftest_wait_timeout")
 
 
 STATIC_ARENA_BYTES = 4 << 20

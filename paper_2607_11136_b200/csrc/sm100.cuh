@@ -83,7 +83,8 @@ __device__ __forceinline__ bool mbar_peek(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-static __device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag) {
+static __device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                                   long long limit_cycles) {
   const long long t0 = clock64();
   uint32_t polls = 0;
   while (true) {
@@ -100,7 +101,7 @@ static __device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parit
     if (ok) return true;
     if ((++polls & 0x3F) == 0) {
       if (*abort_flag) return false;
-      if (clock64() - t0 > kWaitLimitCycles) {
+      if (clock64() - t0 > limit_cycles) {
         *abort_flag = 1;
         return false;
       }
@@ -112,7 +113,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
 #pragma unroll 1
   for (int i = 0; i < XEMA_WAIT_FAST_POLLS; ++i)
     if (mbar_test(bar, parity)) return true;
-  return mbar_wait_slow(bar, parity, abort_flag);
+  return mbar_wait_slow(bar, parity, abort_flag, kWaitLimitCycles);
 }
 
 // ---- fences ----------------------------------------------------------------------------

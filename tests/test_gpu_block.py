@@ -219,3 +219,30 @@ def test_full_size_block_sampled_rows(name):
             assert np.array_equal(first, y), C
         del s
         torch.cuda.empty_cache()
+
+
+def test_bounded_wait_gives_up_and_reports():
+    """A wait on a barrier nothing completes runs out after its limit, sets the status word and
+    leaves the context usable (the next forward call still matches the oracle)."""
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    waited = torch.zeros(1, dtype=torch.int64, device=DEV)
+    limit = 2_000_000                                   # about a millisecond of SM cycles
+    xb.xema_selftest_wait_timeout(status.data_ptr(), limit, waited.data_ptr())
+    torch.cuda.synchronize()
+    assert (int(status.item()) & 0xFFFFFFFF) == xb.DEVICE_STATUS_TIMEOUT
+    assert limit <= int(waited.item()) < 50 * limit
+    # the session turns a non-zero status word into an error ...
+    t = template("tiny")
+    w = make_block_weights(t, 0)
+    x, temb = make_activations(t)
+    s = BlockSession(t, [w], chunks=1)
+    s.status.copy_(status)
+    with pytest.raises(xb.XemaError) as e:
+        s.check_status()
+    assert e.value.status == xb.XEMA_ETIMEOUT
+    # ... and the context is still good for real work
+    s.status.zero_()
+    s.set_inputs(x, temb)
+    s.forward()
+    ref = ob.block_forward(t, _f64(w), bits_to_f64(x), bits_to_f64(temb))["y"]
+    assert_close(bits_to_f64(s.output_bits()), ref, "block after a timed-out wait")
