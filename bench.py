@@ -221,7 +221,8 @@ def main():
     weights = [make_block_weights(t, l) for l in range(t.n_blocks)]
     x_bits, temb_bits = make_activations(t)
     sess = BlockSession(t, weights, chunks=args.chunks or None, budget_bytes=budget, device=dev)
-    n_launch = sess.plan.launch_count()
+    n_launch = sess.plan.n_ops            # logical ops of the trace (fused ones launch nothing)
+    n_kernels = sess.plan.launch_count()  # kernels actually launched per step
     ops = [sess.plan.op(i) for i in range(n_launch)]
     flops = block_flops(t)
     stream = torch.cuda.current_stream(dev)
@@ -357,7 +358,7 @@ def main():
         "clocks": clocks,
         "e2e": {"value": whole_job_tflops(flops, world, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
-        "gpu_launches": n_launch * args.steps,
+        "gpu_launches": n_kernels * args.steps,
         "roofline": roofline,
         "tensor_ops": {"tflops": tensor_fl / (tensor_ms * 1e-3) / 1e12, "ms": tensor_ms,
                        "frac_of_sustained": tensor_fl / (tensor_ms * 1e-3) / 1e12 / peaks["bf16_sustained"],

@@ -242,7 +242,11 @@ enum {
   XEMA_EPI_BIAS = 0,       /* out bf16 = acc + bias                                        */
   XEMA_EPI_BIAS_GELU = 1,  /* out bf16 = gelu_tanh(acc + bias)                             */
   XEMA_EPI_GATE_RES_F32 = 2,  /* out fp32 = resid(bf16) + gate[b,:] * (acc + bias)         */
-  XEMA_EPI_GATE_RES_BF16 = 3  /* out bf16 = resid(fp32) + gate[b,:] * (acc + bias)         */
+  XEMA_EPI_GATE_RES_BF16 = 3, /* out bf16 = resid(fp32) + gate[b,:] * (acc + bias)         */
+  XEMA_EPI_BIAS_NORM_ROPE = 4 /* out bf16 = acc + bias; heads that start below column
+                                 norm_cols additionally get RoPE(RMSNorm(.) * norm_gain), the
+                                 same arithmetic as xema_op_rmsnorm_rope but on the fp32
+                                 accumulator (one rounding less).  Needs N % 256 == 0.        */
 };
 typedef struct xema_gemm_args {
   const void* a;        /* device bf16, row (b,i) at element (b*a_batch_rows + i)*lda      */
@@ -258,6 +262,14 @@ typedef struct xema_gemm_args {
   int64_t gate_stride;
   int32_t batch, rows, N, K; /* N % 128 == 0, K % 64 == 0                                  */
   int32_t epilogue;     /* XEMA_EPI_*                                                      */
+  /* XEMA_EPI_BIAS_NORM_ROPE only (ignored otherwise): */
+  int32_t head_dim;     /* 64 or 128                                                       */
+  int32_t norm_cols;    /* multiple of head_dim, <= N: columns [0, norm_cols) are heads to
+                           normalise and rotate (D for a K|V product, N for a Q product)   */
+  int32_t rope_pos0;    /* token index of row 0: row i uses table row rope_pos0 + i        */
+  float rms_eps;
+  const void* norm_gain; /* device bf16 [head_dim]                                          */
+  const float* rope;     /* device fp32 [tokens][head_dim/2][cos, sin]                      */
 } xema_gemm_args;
 int xema_op_gemm(const xema_gemm_args* args, void* status_dev, void* stream);
 

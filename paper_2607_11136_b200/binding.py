@@ -16,7 +16,7 @@ LIB_PATH = os.environ.get("XEMA_LIB") or os.path.join(_HERE, "libxema.so")
 
 XEMA_OK, XEMA_EINVAL, XEMA_ENOSPC, XEMA_EBUDGET = 0, -1, -2, -3
 XEMA_EALIGN, XEMA_ECUDA, XEMA_ETIMEOUT, XEMA_ESTATE = -4, -5, -6, -7
-EPI_BIAS, EPI_BIAS_GELU, EPI_GATE_RES_F32, EPI_GATE_RES_BF16 = 0, 1, 2, 3
+EPI_BIAS, EPI_BIAS_GELU, EPI_GATE_RES_F32, EPI_GATE_RES_BF16, EPI_BIAS_NORM_ROPE = 0, 1, 2, 3, 4
 
 EXPORTS = (
     "xema_trace", "xema_plan_arena", "xema_chunks_for_budget", "xema_rope_table",
@@ -63,7 +63,9 @@ class xema_gemm_args(C.Structure):
                 ("resid", C.c_void_p), ("ldr", C.c_int64), ("resid_batch_rows", C.c_int64),
                 ("gate", C.c_void_p), ("gate_stride", C.c_int64),
                 ("batch", C.c_int32), ("rows", C.c_int32), ("N", C.c_int32), ("K", C.c_int32),
-                ("epilogue", C.c_int32)]
+                ("epilogue", C.c_int32), ("head_dim", C.c_int32), ("norm_cols", C.c_int32),
+                ("rope_pos0", C.c_int32), ("rms_eps", C.c_float), ("norm_gain", C.c_void_p),
+                ("rope", C.c_void_p)]
 
 
 _lib = None

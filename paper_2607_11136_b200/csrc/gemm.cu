@@ -45,6 +45,12 @@ struct GemmParams {
   long long gate_stride;
   int batch, rows, N, K;
   unsigned int* status;
+  // XEMA_EPI_BIAS_NORM_ROPE only: heads that start below column norm_cols get RMSNorm * gain
+  // and RoPE in the epilogue (a thread owns whole rows, hence whole heads, of the tile)
+  const __nv_bfloat16* norm_gain;   // [head_dim]
+  const float* rope;                // [token][head_dim/2][cos, sin]
+  int rope_pos0, head_dim, norm_cols;
+  float rms_eps;
 };
 
 __device__ __forceinline__ float gelu_tanh_f(float z) {
@@ -112,6 +118,51 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, int b, int r
             pack_bf16x2(fmaf(g1.z, v[8 * q + 6], x1.z), fmaf(g1.w, v[8 * q + 7], x1.w)));
       }
     }
+  }
+}
+
+// One head (DH columns starting at n0) of this thread's row: acc + bias, RMSNorm over the head,
+// gain, rotation of adjacent pairs by the token's angles, bf16 store.
+template <int DH>
+__device__ __forceinline__ void epilogue_head_norm_rope(const GemmParams& p, int b, int row, int n0, uint32_t t_cols) {
+  float v[DH];
+#pragma unroll
+  for (int ch = 0; ch < DH / 32; ++ch)
+    tmem_ld32(t_cols + ch * 32, *reinterpret_cast<uint32_t(*)[32]>(&v[ch * 32]));
+  tmem_ld_wait();
+  if (row >= p.rows) return;
+  float ss = 0.f;
+#pragma unroll
+  for (int q = 0; q < DH / 8; ++q) {
+    const uint4 bb = __ldg(reinterpret_cast<const uint4*>(p.bias + n0) + q);
+    v[8 * q + 0] += bf16_lo(bb.x); v[8 * q + 1] += bf16_hi(bb.x);
+    v[8 * q + 2] += bf16_lo(bb.y); v[8 * q + 3] += bf16_hi(bb.y);
+    v[8 * q + 4] += bf16_lo(bb.z); v[8 * q + 5] += bf16_hi(bb.z);
+    v[8 * q + 6] += bf16_lo(bb.w); v[8 * q + 7] += bf16_hi(bb.w);
+#pragma unroll
+    for (int t = 0; t < 8; ++t) ss = fmaf(v[8 * q + t], v[8 * q + t], ss);
+  }
+  const float rstd = rsqrtf(ss * (1.f / DH) + p.rms_eps);
+  const float4* rp = reinterpret_cast<const float4*>(p.rope + (size_t)(p.rope_pos0 + row) * DH);
+  uint4* op = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.out) +
+                                       ((size_t)b * p.out_batch_rows + row) * p.ldo + n0);
+#pragma unroll
+  for (int q = 0; q < DH / 8; ++q) {
+    const uint4 gg = __ldg(reinterpret_cast<const uint4*>(p.norm_gain) + q);
+    const float gn[8] = {bf16_lo(gg.x), bf16_hi(gg.x), bf16_lo(gg.y), bf16_hi(gg.y),
+                         bf16_lo(gg.z), bf16_hi(gg.z), bf16_lo(gg.w), bf16_hi(gg.w)};
+    const float4 cs0 = __ldg(rp + 2 * q), cs1 = __ldg(rp + 2 * q + 1);
+    const float cosv[4] = {cs0.x, cs0.z, cs1.x, cs1.z};
+    const float sinv[4] = {cs0.y, cs0.w, cs1.y, cs1.w};
+    float y[8];
+#pragma unroll
+    for (int pr = 0; pr < 4; ++pr) {
+      const float a = v[8 * q + 2 * pr] * rstd * gn[2 * pr];
+      const float c = v[8 * q + 2 * pr + 1] * rstd * gn[2 * pr + 1];
+      y[2 * pr] = a * cosv[pr] - c * sinv[pr];
+      y[2 * pr + 1] = a * sinv[pr] + c * cosv[pr];
+    }
+    op[q] = make_uint4(pack_bf16x2(y[0], y[1]), pack_bf16x2(y[2], y[3]), pack_bf16x2(y[4], y[5]), pack_bf16x2(y[6], y[7]));
   }
 }
 
@@ -258,12 +309,32 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
       tc_fence_after();
       const int row = c.mt * BM + quad * 32 + lane;
       const uint32_t t_addr = tmem_base + ((uint32_t)(quad * 32) << 16) + acc * BN;
+      if constexpr (EPI == XEMA_EPI_BIAS_NORM_ROPE) {
+        // head by head; heads at or beyond norm_cols (the V half of a KV product) get the bias only
 #pragma unroll 1
-      for (int ch = 0; ch < BN / 32; ++ch) {
-        uint32_t r[32];
-        tmem_ld32(t_addr + ch * 32, r);
-        tmem_ld_wait();
-        epilogue_chunk<EPI>(p, c.b, row, c.nt * BN + ch * 32, r);
+        for (int hc = 0; hc < BN; hc += p.head_dim) {
+          const int n0 = c.nt * BN + hc;
+          if (n0 < p.norm_cols) {
+            if (p.head_dim == 64) epilogue_head_norm_rope<64>(p, c.b, row, n0, t_addr + hc);
+            else epilogue_head_norm_rope<128>(p, c.b, row, n0, t_addr + hc);
+          } else {
+#pragma unroll 1
+            for (int ch = 0; ch < p.head_dim / 32; ++ch) {
+              uint32_t r[32];
+              tmem_ld32(t_addr + hc + ch * 32, r);
+              tmem_ld_wait();
+              epilogue_chunk<XEMA_EPI_BIAS>(p, c.b, row, n0 + ch * 32, r);
+            }
+          }
+        }
+      } else {
+#pragma unroll 1
+        for (int ch = 0; ch < BN / 32; ++ch) {
+          uint32_t r[32];
+          tmem_ld32(t_addr + ch * 32, r);
+          tmem_ld_wait();
+          epilogue_chunk<EPI>(p, c.b, row, c.nt * BN + ch * 32, r);
+        }
       }
       tc_fence_before();
       __syncwarp();
@@ -322,6 +393,12 @@ static int launch_gemm_t(const GemmLaunch& g, cudaStream_t stream) {
   p.N = g.N;
   p.K = g.K;
   p.status = g.status;
+  p.norm_gain = (const __nv_bfloat16*)g.norm_gain;
+  p.rope = g.rope;
+  p.rope_pos0 = g.rope_pos0;
+  p.head_dim = g.head_dim;
+  p.norm_cols = g.norm_cols;
+  p.rms_eps = g.rms_eps;
   const int m_tiles = (g.rows + BM - 1) / BM;
   const long long tiles = (long long)g.batch * m_tiles * (g.N / BN);
   const int grid = (int)std::min<long long>(tiles, sm_count());
@@ -336,6 +413,7 @@ static int launch_gemm_bn(const GemmLaunch& g, cudaStream_t stream) {
     case XEMA_EPI_BIAS_GELU: return launch_gemm_t<BN, XEMA_EPI_BIAS_GELU>(g, stream);
     case XEMA_EPI_GATE_RES_F32: return launch_gemm_t<BN, XEMA_EPI_GATE_RES_F32>(g, stream);
     case XEMA_EPI_GATE_RES_BF16: return launch_gemm_t<BN, XEMA_EPI_GATE_RES_BF16>(g, stream);
+    case XEMA_EPI_BIAS_NORM_ROPE: return launch_gemm_t<BN, XEMA_EPI_BIAS_NORM_ROPE>(g, stream);
     default: return XEMA_EINVAL;
   }
 }
@@ -349,11 +427,17 @@ int launch_gemm(const GemmLaunch& g, cudaStream_t stream) {
 
 int gemm_prepare(GemmLaunch* g, const void* a, long long lda, long long a_batch_rows, const void* w, long long ldw) {
   if (g->batch < 1 || g->rows < 0 || g->N < 128 || (g->N % 128) || g->K < 64 || (g->K % 64)) return XEMA_EINVAL;
-  if (g->epilogue < XEMA_EPI_BIAS || g->epilogue > XEMA_EPI_GATE_RES_BF16) return XEMA_EINVAL;
+  if (g->epilogue < XEMA_EPI_BIAS || g->epilogue > XEMA_EPI_BIAS_NORM_ROPE) return XEMA_EINVAL;
   if (!a || !w || !g->bias || !g->out) return XEMA_EINVAL;
-  if (g->epilogue >= XEMA_EPI_GATE_RES_F32 && (!g->resid || !g->gate)) return XEMA_EINVAL;
-  if ((lda & 7) || (ldw & 7) || (g->ldo & 7) || (g->epilogue >= XEMA_EPI_GATE_RES_F32 && (g->ldr & 7)))
-    return XEMA_EALIGN;
+  const bool gated = g->epilogue == XEMA_EPI_GATE_RES_F32 || g->epilogue == XEMA_EPI_GATE_RES_BF16;
+  if (gated && (!g->resid || !g->gate)) return XEMA_EINVAL;
+  if (g->epilogue == XEMA_EPI_BIAS_NORM_ROPE) {
+    if (!g->norm_gain || !g->rope || (g->head_dim != 64 && g->head_dim != 128)) return XEMA_EINVAL;
+    if (g->norm_cols < 0 || g->norm_cols > g->N || g->norm_cols % g->head_dim || g->N % 256 || g->rope_pos0 < 0)
+      return XEMA_EINVAL;
+    if ((reinterpret_cast<uintptr_t>(g->norm_gain) & 15) || (reinterpret_cast<uintptr_t>(g->rope) & 15)) return XEMA_EALIGN;
+  }
+  if ((lda & 7) || (ldw & 7) || (g->ldo & 7) || (gated && (g->ldr & 7))) return XEMA_EALIGN;
   auto mis = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) != 0; };
   if (mis(a) || mis(w) || mis(g->bias) || mis(g->out) || (g->resid && mis(g->resid)) || (g->gate && mis(g->gate)))
     return XEMA_EALIGN;

@@ -39,6 +39,11 @@ struct GemmLaunch {
   long long gate_stride;
   int batch, rows, N, K, epilogue, block_n;
   unsigned int* status;
+  // XEMA_EPI_BIAS_NORM_ROPE: RMSNorm * gain + RoPE for the heads below column norm_cols
+  const void* norm_gain;
+  const float* rope;
+  int rope_pos0, head_dim, norm_cols;
+  float rms_eps;
 };
 // Fills map_a / map_w / block_n from plain pointers.
 int gemm_prepare(GemmLaunch* g, const void* a, long long lda, long long a_batch_rows, const void* w, long long ldw);

@@ -28,7 +28,7 @@ def test_struct_sizes_match_the_header():
     assert ctypes.sizeof(xb.xema_config) == 68
     assert ctypes.sizeof(xb.xema_tensor) == 56
     assert ctypes.sizeof(xb.xema_block_weights) == 96
-    assert ctypes.sizeof(xb.xema_gemm_args) == 136
+    assert ctypes.sizeof(xb.xema_gemm_args) == 168
 
 
 def test_error_paths_without_gpu():

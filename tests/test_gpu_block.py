@@ -111,7 +111,7 @@ def test_forward_stays_inside_the_planned_arena(tiny_case):
     s.forward()
     torch.cuda.synchronize()
     assert bool((arena[plan.peak_bytes:] == 0x5A).all())
-    assert s.plan.launch_count() == s.plan.n_ops == 23
+    assert s.plan.n_ops == 23 and s.plan.launch_count() == 23 - 2 * 2      # KROPE, QROPE run inside the GEMMs
     # the forward call itself allocated nothing on the device
     free1, _ = torch.cuda.mem_get_info()
     s.forward()

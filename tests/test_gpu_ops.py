@@ -229,3 +229,35 @@ def test_attention_rows_are_chunk_invariant():
     _sync_status(status)
     assert torch.equal(o_all[:, 167:167 + 211], o_part)
     assert torch.equal(l_all[:, :, 167:167 + 211], l_part)
+
+
+@pytest.mark.parametrize("name,norm_all", [("tiny", True), ("tiny", False), ("flux", True), ("flux", False)])
+def test_gemm_epilogue_rmsnorm_rope(name, norm_all):
+    """Linear + per-head RMSNorm * gain + RoPE fused in the GEMM epilogue: the Q product
+    (every head) and the K|V product (heads of the first half only)."""
+    t = template(name)
+    dh = t.head_dim
+    rng = np.random.default_rng(31 + dh + norm_all)
+    H, K, rows, pos0, B = 4, 192, 200, t.s_text - 20, 2         # rows span the text / video boundary
+    Dh = H * dh
+    N = Dh if norm_all else 2 * Dh
+    ab, af = rand_bf16(rng, (B, rows, K))
+    wb, wf = rand_bf16(rng, (N, K), 0.08)
+    bb, bf = rand_bf16(rng, (N,), 0.3)
+    gb, gf = rand_bf16(rng, (dh,), 1.0)
+    a_dev, w_dev, b_dev, g_dev = to_dev(ab), to_dev(wb), to_dev(bb), to_dev(gb)
+    rope = torch.from_numpy(xb.xema_rope_table(xb.make_config(t))).to(DEV)
+    out = torch.full((B, rows, N), 0x7FC0, dtype=torch.int16, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    xb.xema_op_gemm(status=status.data_ptr(), a=a_dev.data_ptr(), lda=K, a_batch_rows=rows, w=w_dev.data_ptr(), ldw=K,
+                    bias=b_dev.data_ptr(), out=out.data_ptr(), ldo=N, out_batch_rows=rows, batch=B, rows=rows, N=N,
+                    K=K, epilogue=xb.EPI_BIAS_NORM_ROPE, head_dim=dh, norm_cols=Dh, rope_pos0=pos0, rms_eps=1e-6,
+                    norm_gain=g_dev.data_ptr(), rope=rope.data_ptr())
+    _sync_status(status)
+    acc = af @ wf.T + bf
+    ang = ob.rope_angles(t)[pos0:pos0 + rows]
+    ref = acc.copy()
+    for b in range(B):
+        v = acc[b, :, :Dh].reshape(rows, H, dh)
+        ref[b, :, :Dh] = ob.apply_rope(ob.rms_norm(v, gf, 1e-6), ang).reshape(rows, Dh)
+    assert_bf16_close(from_dev_bf16(out), ref, ("gemm norm+rope", name, norm_all), atol_rms=3e-4)
