@@ -15,6 +15,9 @@
  *   xema_chunks_for_budget  smallest chunk count whose reserved peak fits the budget
  *                           (section "Applying Only as Much Mitigation as Needed", with the
  *                           chunk count as the mitigation intensity; "Localized chunking")
+ *   xema_phase_chunks_for_budget  one chunk count per phase of the block, raised only in
+ *                           the phases whose trace exceeds the budget (section "Applying
+ *                           Mitigation Only Where Needed")
  *   xema_block_forward /    run one block / all n_blocks blocks on a caller-given CUDA
  *   xema_step_forward       stream over caller-owned arena memory ("Static memory
  *                           runtime": allocation at run time is a table lookup)
@@ -129,6 +132,28 @@ int xema_plan_arena(const xema_tensor* tensors, size_t n, uint64_t* offsets,
 int xema_chunks_for_budget(const xema_config* cfg, uint64_t budget_bytes, int32_t max_chunks,
                            int32_t* chunks, uint64_t* peak_bytes);
 
+/* Per-phase chunk counts (section "Applying Mitigation Only Where Needed": the planner
+ * locates, on the memory trace, where the budget is exceeded and mitigates only there).
+ * A block has three phases: 0 = keys/values (LN1A, KV, KROPE per chunk), 1 = queries,
+ * attention, output projection (LN1B, Q, QROPE, ATTN, PROJ per chunk), 2 = feed-forward
+ * (LN2, FFN1, FFN2 per chunk).  chunks[3] (host) holds one count per phase; phase p splits
+ * the S rows into chunks[p] pieces by the rule above; a block then has
+ * 1 + 3*chunks[0] + 5*chunks[1] + 3*chunks[2] ops.  Otherwise as xema_trace, which is the
+ * case chunks[0] = chunks[1] = chunks[2]. */
+int xema_trace_phases(const xema_config* cfg, const int32_t chunks[3], xema_tensor* out,
+                      size_t cap, size_t* n_tensors, uint32_t* n_ops);
+
+/* Search for per-phase counts that fit: start at (1, 1, 1); on the trace of the current
+ * counts, every phase that holds an op whose live bytes exceed budget_bytes gets one more
+ * chunk; repeat.  When no op is over, the trace is laid out (Algorithm 1); if the reserved
+ * peak still exceeds the budget, the phase holding the op with the most live bytes (lowest
+ * op index on ties) gets one more chunk.  chunks (host, 3 entries) receives the counts and
+ * *peak_bytes the reserved peak.  XEMA_EBUDGET when a phase would need more than
+ * min(max_chunks, S) chunks: chunks is then zeroed and *peak_bytes is the smallest reserved
+ * peak seen. */
+int xema_phase_chunks_for_budget(const xema_config* cfg, uint64_t budget_bytes,
+                                 int32_t max_chunks, int32_t chunks[3], uint64_t* peak_bytes);
+
 /* RoPE table for the template: host_out (host) receives S * (dh/2) * 2 floats laid out
  * [token][pair][cos, sin]; angle = position * rope_base^(-2j/d) inside each of the three
  * sections (t, h, w), evaluated in double precision and rounded once.  Text tokens sit at
@@ -141,11 +166,16 @@ typedef struct xema_plan xema_plan; /* opaque; host memory owned by the library 
 
 /* Traces and lays out the template for `chunks` chunks.  No CUDA call. */
 int xema_plan_create(const xema_config* cfg, int32_t chunks, xema_plan** out);
+/* The same with one chunk count per phase (see xema_trace_phases). */
+int xema_plan_create_phases(const xema_config* cfg, const int32_t chunks[3], xema_plan** out);
 void xema_plan_destroy(xema_plan* plan);
 
-/* Plan figures: any output pointer may be NULL. */
+/* Plan figures: any output pointer may be NULL.  *chunks is the largest of the plan's three
+ * per-phase counts (the count itself for a plan made by xema_plan_create). */
 int xema_plan_info(const xema_plan* plan, uint64_t* peak_bytes, uint64_t* max_live_bytes,
                    size_t* n_tensors, uint32_t* n_ops, int32_t* chunks);
+/* The plan's per-phase chunk counts; chunks: host, 3 entries. */
+int xema_plan_phase_chunks(const xema_plan* plan, int32_t chunks[3]);
 /* Offset and (256-rounded) size of a tensor by name, e.g. "hid0", "temb", "hid1", "res0". */
 int xema_plan_tensor(const xema_plan* plan, const char* name, uint64_t* offset, uint64_t* bytes);
 /* Copy of the plan's tensor i and its offset. */

@@ -76,6 +76,68 @@ def overlapping_pairs(tensors, offsets):
     return bad
 
 
+def reserved_per_op(tensors, offsets, n_ops):
+    """Reserved-memory trace: for every op, the highest address used by a tensor live at it."""
+    out = [0] * n_ops
+    for d, off in zip(tensors, offsets):
+        top = off + d["bytes"]
+        for op in range(d["birth"], d["death"]):
+            if top > out[op]:
+                out[op] = top
+    return out
+
+
+def phase_of_op(t, counts, op):
+    """0 / 1 / 2 for an op of the key-value / attention / feed-forward phase of its block; the
+    MOD op belongs to phase 0."""
+    ca, cb, cc = counts
+    per_block = 1 + 3 * ca + 5 * cb + 3 * cc
+    k = op % per_block
+    if k < 1 + 3 * ca:
+        return 0
+    if k < 1 + 3 * ca + 5 * cb:
+        return 1
+    return 2
+
+
+def live_per_op(tensors, n_ops):
+    """Active-memory trace: bytes of the tensors live at every op."""
+    out = [0] * n_ops
+    for d in tensors:
+        for op in range(d["birth"], d["death"]):
+            out[op] += d["bytes"]
+    return out
+
+
+def phase_chunks_for_budget(t, budget_bytes, max_chunks):
+    """Mitigation only where it is needed (the planner's stage "locating where memory exceeds
+    the budget", with chunking as the mitigation): start unchunked; mark the phases in which
+    the active-memory trace exceeds the budget at some op; raise the chunk count of exactly
+    those phases by one; repeat until no phase is over.  The trace is then laid out; should the
+    reserved peak still exceed the budget (Algorithm 1 is a heuristic), the phase holding the
+    op with the most live bytes is raised as well.  Returns ((C_A, C_B, C_C), reserved peak),
+    or (None, smallest reserved peak seen) when a phase would need more than max_chunks.
+    (The per-op reserved memory is no guide here: the longest-lived tensors sit at the top of
+    the arena, so every op reaches the peak address.)"""
+    counts = [1, 1, 1]
+    smallest = None
+    limit = min(max_chunks, t.seq)
+    while True:
+        tensors, n_ops = _trace.trace(t, tuple(counts))
+        _, peak = plan_arena(tensors)
+        smallest = peak if smallest is None else min(smallest, peak)
+        live = live_per_op(tensors, n_ops)
+        over = {phase_of_op(t, counts, op) for op, b in enumerate(live) if b > budget_bytes}
+        if not over:
+            if peak <= budget_bytes:
+                return tuple(counts), peak
+            over = {phase_of_op(t, counts, max(range(n_ops), key=lambda op: (live[op], -op)))}
+        for ph in sorted(over):
+            counts[ph] += 1
+            if counts[ph] > limit:
+                return None, smallest
+
+
 def chunks_for_budget(t, budget_bytes, max_chunks):
     """Returns (chunks, peak) for the first C in 1..max_chunks whose arena peak fits,
     or (None, smallest peak seen) when none does."""

@@ -173,12 +173,13 @@ def block_forward(t, W, x, temb, rows=None, row_block=2048, keep=False):
 def block_forward_chunked(t, W, x, temb, chunks):
     """The same block evaluated in the chunked three-phase order the library uses
     (all KV chunks; then Q/attention/projection per chunk; then the FFN per chunk),
-    chunk c covering rows [floor(c S / C), floor((c+1) S / C)).  Used to show that
-    chunking is lossless; not a second definition."""
+    chunk c covering rows [floor(c S / C), floor((c+1) S / C)); `chunks` is one count or
+    a per-phase triple.  Used to show that chunking is lossless; not a second definition."""
     x = np.asarray(x, F64)
     B, S, D = x.shape
     H, dh = t.heads, t.head_dim
-    r = [c * S // chunks for c in range(chunks + 1)]
+    ca, cb, cc = (chunks, chunks, chunks) if isinstance(chunks, int) else chunks
+    rows_of = lambda C: [c * S // C for c in range(C + 1)]
     shift1, scale1, gate1, shift2, scale2, gate2 = modulation(t, W, temb)
     ang = rope_angles(t)
     scale = 1.0 / math.sqrt(dh)
@@ -187,13 +188,15 @@ def block_forward_chunked(t, W, x, temb, chunks):
     for b in range(B):
         k = np.empty((S, H, dh))
         v = np.empty((S, H, dh))
-        for c in range(chunks):
+        r = rows_of(ca)
+        for c in range(ca):
             sl = slice(r[c], r[c + 1])
             h = layer_norm(x[b, sl], t.ln_eps) * (1.0 + scale1[b]) + shift1[b]
             k[sl] = qkv_heads(t, W, h, ang[sl], "k")
             v[sl] = qkv_heads(t, W, h, ang[sl], "v")
         res = np.empty((S, D))
-        for c in range(chunks):
+        r = rows_of(cb)
+        for c in range(cb):
             sl = slice(r[c], r[c + 1])
             h = layer_norm(x[b, sl], t.ln_eps) * (1.0 + scale1[b]) + shift1[b]
             q = qkv_heads(t, W, h, ang[sl], "q")
@@ -201,7 +204,8 @@ def block_forward_chunked(t, W, x, temb, chunks):
             for hd in range(H):
                 o[:, hd], lse[b, hd, sl] = attention_head(q[:, hd], k[:, hd], v[:, hd], scale)
             res[sl] = x[b, sl] + gate1[b] * linear(o.reshape(-1, D), W["w_o"], W["b_o"])
-        for c in range(chunks):
+        r = rows_of(cc)
+        for c in range(cc):
             sl = slice(r[c], r[c + 1])
             h2 = layer_norm(res[sl], t.ln_eps) * (1.0 + scale2[b]) + shift2[b]
             g = gelu_tanh(linear(h2, W["w_1"], W["b_1"]))

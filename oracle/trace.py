@@ -51,15 +51,27 @@ class _Recorder:
         self.t += 1
 
 
+def phase_counts(chunks):
+    """chunks: one count for all three phases, or a triple (C_A, C_B, C_C) for the key/value
+    phase, the query/attention/projection phase and the feed-forward phase."""
+    if isinstance(chunks, int):
+        return (chunks, chunks, chunks)
+    ca, cb, cc = (int(v) for v in chunks)
+    return (ca, cb, cc)
+
+
 def trace(t, chunks):
     """Returns (tensors, n_ops).  tensors: list of dicts with name, kind, dtype, block,
     chunk, bytes (rounded up to 256), birth, death -- in id order (first birth, then
-    table row)."""
+    table row).  `chunks` is an int or a per-phase triple (see phase_counts); with a triple
+    the op list is MOD; C_A x (LN1A, KV, KROPE); C_B x (LN1B, Q, QROPE, ATTN, PROJ);
+    C_C x (LN2, FFN1, FFN2) -- chunking applied only where the trace needs it."""
     B, S, D, H, F, Dt = t.batch, t.seq, t.hidden, t.heads, t.ffn, t.temb_dim
-    C, L = chunks, t.n_blocks
-    if C < 1 or C > S:
+    CA, CB, CC = phase_counts(chunks)
+    L = t.n_blocks
+    if min(CA, CB, CC) < 1 or max(CA, CB, CC) > S:
         raise ValueError("chunks must be in [1, S]")
-    r = chunk_rows(S, C)
+    rA, rB, rC = chunk_rows(S, CA), chunk_rows(S, CB), chunk_rows(S, CC)
     rec = _Recorder()
 
     def meta(base, nbytes, kind, dtype, block, chunk=-1):
@@ -77,14 +89,14 @@ def trace(t, chunks):
         m_res = (res, meta("res", 2 * u, KIND_FULL, DTYPE_F32, l))
         m_nxt = (nxt, meta("hid", u, KIND_OUTPUT if l + 1 == L else KIND_FULL, DTYPE_BF16, l + 1))
         rec.op(reads=["temb"], writes=[m_mod])                                   # MOD
-        for c in range(C):
-            n = r[c + 1] - r[c]
+        for c in range(CA):
+            n = rA[c + 1] - rA[c]
             h1a = (f"h1a{l}_{c}", meta("h1a", 2 * B * n * D, KIND_CHUNK, DTYPE_BF16, l, c))
             rec.op(reads=[hid, mod], writes=[h1a])                               # LN1A
             rec.op(reads=[h1a[0]], writes=[m_kv])                                # KV
             rec.op(reads=[kv], writes=[m_kv])                                    # KROPE (in place)
-        for c in range(C):
-            n = r[c + 1] - r[c]
+        for c in range(CB):
+            n = rB[c + 1] - rB[c]
             h1b = (f"h1b{l}_{c}", meta("h1b", 2 * B * n * D, KIND_CHUNK, DTYPE_BF16, l, c))
             q = (f"q{l}_{c}", meta("q", 2 * B * n * D, KIND_CHUNK, DTYPE_BF16, l, c))
             o = (f"o{l}_{c}", meta("o", 2 * B * n * D, KIND_CHUNK, DTYPE_BF16, l, c))
@@ -94,8 +106,8 @@ def trace(t, chunks):
             rec.op(reads=[q[0]], writes=[q])                                     # QROPE (in place)
             rec.op(reads=[q[0], kv], writes=[o, lse])                            # ATTN
             rec.op(reads=[o[0], hid, mod], writes=[m_res])                       # PROJ
-        for c in range(C):
-            n = r[c + 1] - r[c]
+        for c in range(CC):
+            n = rC[c + 1] - rC[c]
             h2 = (f"h2{l}_{c}", meta("h2", 2 * B * n * D, KIND_CHUNK, DTYPE_BF16, l, c))
             g = (f"g{l}_{c}", meta("g", 2 * B * n * F, KIND_CHUNK, DTYPE_BF16, l, c))
             rec.op(reads=[res, mod], writes=[h2])                                # LN2

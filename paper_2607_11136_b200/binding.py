@@ -19,8 +19,10 @@ XEMA_EALIGN, XEMA_ECUDA, XEMA_ETIMEOUT, XEMA_ESTATE = -4, -5, -6, -7
 EPI_BIAS, EPI_BIAS_GELU, EPI_GATE_RES_F32, EPI_GATE_RES_BF16, EPI_BIAS_NORM_ROPE = 0, 1, 2, 3, 4
 
 EXPORTS = (
-    "xema_trace", "xema_plan_arena", "xema_chunks_for_budget", "xema_rope_table",
-    "xema_plan_create", "xema_plan_destroy", "xema_plan_info", "xema_plan_tensor",
+    "xema_trace", "xema_trace_phases", "xema_plan_arena", "xema_chunks_for_budget",
+    "xema_phase_chunks_for_budget", "xema_rope_table",
+    "xema_plan_create", "xema_plan_create_phases", "xema_plan_destroy", "xema_plan_info",
+    "xema_plan_phase_chunks", "xema_plan_tensor",
     "xema_plan_tensor_at", "xema_plan_bind", "xema_block_forward", "xema_step_forward",
     "xema_block_forward_static",
     "xema_plan_launch_count", "xema_forward_prefix", "xema_forward_range", "xema_plan_op", "xema_op_mod", "xema_op_ln_modulate",
@@ -83,6 +85,10 @@ def lib() -> C.CDLL:
         P = C.POINTER
         sig = {
             "xema_trace": [P(xema_config), i32, P(xema_tensor), sz, P(sz), P(u32)],
+            "xema_trace_phases": [P(xema_config), P(i32), P(xema_tensor), sz, P(sz), P(u32)],
+            "xema_phase_chunks_for_budget": [P(xema_config), u64, i32, P(i32), P(u64)],
+            "xema_plan_create_phases": [P(xema_config), P(i32), P(vp)],
+            "xema_plan_phase_chunks": [vp, P(i32)],
             "xema_plan_arena": [P(xema_tensor), sz, P(u64), P(u64), P(u64)],
             "xema_chunks_for_budget": [P(xema_config), u64, i32, P(i32), P(u64)],
             "xema_rope_table": [P(xema_config), vp],
@@ -161,6 +167,33 @@ def xema_trace(cfg: xema_config, chunks: int):
     return [_tensor_dict(t) for t in arr], ops.value
 
 
+def _triple(chunks):
+    ca, cb, cc = (int(v) for v in chunks)
+    return (C.c_int32 * 3)(ca, cb, cc)
+
+
+def xema_trace_phases(cfg: xema_config, chunks):
+    """chunks = (C_A, C_B, C_C) -> (list of tensor dicts in id order, n_ops)"""
+    c3 = _triple(chunks)
+    n, ops = C.c_size_t(0), C.c_uint32(0)
+    rc = lib().xema_trace_phases(C.byref(cfg), c3, None, 0, C.byref(n), C.byref(ops))
+    if rc != XEMA_ENOSPC:
+        _check(rc, "xema_trace_phases")
+    arr = (xema_tensor * n.value)()
+    _check(lib().xema_trace_phases(C.byref(cfg), c3, arr, n.value, C.byref(n), C.byref(ops)), "xema_trace_phases")
+    return [_tensor_dict(t) for t in arr], ops.value
+
+
+def xema_phase_chunks_for_budget(cfg: xema_config, budget_bytes: int, max_chunks: int):
+    """-> ((C_A, C_B, C_C), peak_bytes); the triple is None when nothing fits."""
+    c3, peak = (C.c_int32 * 3)(), C.c_uint64(0)
+    rc = lib().xema_phase_chunks_for_budget(C.byref(cfg), budget_bytes, max_chunks, c3, C.byref(peak))
+    if rc == XEMA_EBUDGET:
+        return None, peak.value
+    _check(rc, "xema_phase_chunks_for_budget")
+    return tuple(c3), peak.value
+
+
 def xema_plan_arena(tensors: Sequence[dict]):
     """tensors: dicts with bytes, birth, death -> (offsets, peak_bytes, max_live_bytes)"""
     n = len(tensors)
@@ -193,15 +226,23 @@ def xema_rope_table(cfg: xema_config) -> np.ndarray:
 class Plan:
     """Owner of an xema_plan handle."""
 
-    def __init__(self, cfg: xema_config, chunks: int):
+    def __init__(self, cfg: xema_config, chunks):
+        """chunks: one count (xema_plan_create) or a per-phase triple (xema_plan_create_phases)."""
         self.cfg = cfg
         self._h = C.c_void_p()
-        _check(lib().xema_plan_create(C.byref(cfg), chunks, C.byref(self._h)), "xema_plan_create")
+        if isinstance(chunks, int):
+            _check(lib().xema_plan_create(C.byref(cfg), chunks, C.byref(self._h)), "xema_plan_create")
+        else:
+            _check(lib().xema_plan_create_phases(C.byref(cfg), _triple(chunks), C.byref(self._h)),
+                   "xema_plan_create_phases")
         peak, live, n, ops, ch = C.c_uint64(), C.c_uint64(), C.c_size_t(), C.c_uint32(), C.c_int32()
         _check(lib().xema_plan_info(self._h, C.byref(peak), C.byref(live), C.byref(n), C.byref(ops), C.byref(ch)),
                "xema_plan_info")
         self.peak_bytes, self.max_live_bytes = peak.value, live.value
         self.n_tensors, self.n_ops, self.chunks = n.value, ops.value, ch.value
+        c3 = (C.c_int32 * 3)()
+        _check(lib().xema_plan_phase_chunks(self._h, c3), "xema_plan_phase_chunks")
+        self.phase_chunks = tuple(c3)
         self._keep = None
 
     def close(self):

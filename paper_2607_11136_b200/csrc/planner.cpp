@@ -32,20 +32,19 @@ int64_t seq_len(const xema_config& c) {
 // Index of a logical op inside block l.  Phase A holds 3 ops per chunk, phase B 5, phase C 3.
 struct OpIndex {
   uint32_t base;  // index of MOD of this block
-  uint32_t C;
+  uint32_t CA, CB, CC;  // chunks of the key/value, attention and feed-forward phases
   uint32_t mod() const { return base; }
   uint32_t ln1a(uint32_t c) const { return base + 1 + 3 * c; }
   uint32_t kv(uint32_t c) const { return ln1a(c) + 1; }
   uint32_t krope(uint32_t c) const { return ln1a(c) + 2; }
-  uint32_t ln1b(uint32_t c) const { return base + 1 + 3 * C + 5 * c; }
+  uint32_t ln1b(uint32_t c) const { return base + 1 + 3 * CA + 5 * c; }
   uint32_t q(uint32_t c) const { return ln1b(c) + 1; }
   uint32_t qrope(uint32_t c) const { return ln1b(c) + 2; }
   uint32_t attn(uint32_t c) const { return ln1b(c) + 3; }
   uint32_t proj(uint32_t c) const { return ln1b(c) + 4; }
-  uint32_t ln2(uint32_t c) const { return base + 1 + 8 * C + 3 * c; }
+  uint32_t ln2(uint32_t c) const { return base + 1 + 3 * CA + 5 * CB + 3 * c; }
   uint32_t ffn1(uint32_t c) const { return ln2(c) + 1; }
   uint32_t ffn2(uint32_t c) const { return ln2(c) + 2; }
-  uint32_t end() const { return base + 1 + 11 * C; }
 };
 
 static xema_tensor make(const char* stem, int block, int chunk, uint32_t kind, uint32_t dtype,
@@ -69,55 +68,63 @@ static xema_tensor make(const char* stem, int block, int chunk, uint32_t kind, u
 }
 
 int build_trace(const xema_config& cfg, int32_t chunks, std::vector<xema_tensor>& out, uint32_t* n_ops) {
+  const int32_t c3[3] = {chunks, chunks, chunks};
+  return build_trace(cfg, c3, out, n_ops);
+}
+
+int build_trace(const xema_config& cfg, const int32_t chunks[3], std::vector<xema_tensor>& out, uint32_t* n_ops) {
   int rc = validate_config(cfg);
   if (rc) return rc;
   const int64_t S = seq_len(cfg);
-  if (chunks < 1 || chunks > S) return XEMA_EINVAL;
+  for (int i = 0; i < 3; ++i)
+    if (chunks[i] < 1 || chunks[i] > S) return XEMA_EINVAL;
   const uint64_t B = cfg.batch, D = cfg.hidden, H = cfg.heads, F = cfg.ffn, Dt = cfg.temb_dim;
-  const uint32_t C = (uint32_t)chunks, L = (uint32_t)cfg.n_blocks;
-  const uint32_t ops_per_block = 1 + 11 * C;
+  const uint32_t CA = (uint32_t)chunks[0], CB = (uint32_t)chunks[1], CC = (uint32_t)chunks[2];
+  const uint32_t L = (uint32_t)cfg.n_blocks;
+  const uint32_t ops_per_block = 1 + 3 * CA + 5 * CB + 3 * CC;
   const uint32_t total_ops = L * ops_per_block;
   const uint64_t u = 2 * B * (uint64_t)S * D;
+  auto rows_of = [&](uint32_t c, uint32_t C) { return (uint64_t)((int64_t)(c + 1) * S / C - (int64_t)c * S / C); };
 
   out.clear();
-  out.reserve((size_t)L * (4 + 7 * C) + 2);
+  out.reserve((size_t)L * (4 + 2 * CA + 4 * CB + 2 * CC) + 2);
   // Emitted directly in id order: ascending birth; tensors born at the same op follow the
   // order temb, hid, mod, kv, h1a, h1b, q, o, lse, res, h2, g.
-  OpIndex last{(L - 1) * ops_per_block, C};
+  OpIndex last{(L - 1) * ops_per_block, CA, CB, CC};
   out.push_back(make("temb", -1, -1, XEMA_KIND_INPUT, XEMA_DTYPE_BF16, 2 * B * Dt, 0, last.mod() + 1));
   for (uint32_t l = 0; l < L; ++l) {
-    OpIndex op{l * ops_per_block, C};
+    OpIndex op{l * ops_per_block, CA, CB, CC};
     if (l == 0) {
       // the block input is read by LN1A/LN1B and as the residual of PROJ
       uint32_t kind = XEMA_KIND_INPUT;
-      out.push_back(make("hid", 0, -1, kind, XEMA_DTYPE_BF16, u, 0, op.proj(C - 1) + 1));
+      out.push_back(make("hid", 0, -1, kind, XEMA_DTYPE_BF16, u, 0, op.proj(CB - 1) + 1));
     }
-    out.push_back(make("mod", l, -1, XEMA_KIND_FULL, XEMA_DTYPE_F32, 24 * B * D, op.mod(), op.ffn2(C - 1) + 1));
-    for (uint32_t c = 0; c < C; ++c) {
-      uint64_t n = (uint64_t)((int64_t)(c + 1) * S / C - (int64_t)c * S / C);
+    out.push_back(make("mod", l, -1, XEMA_KIND_FULL, XEMA_DTYPE_F32, 24 * B * D, op.mod(), op.ffn2(CC - 1) + 1));
+    for (uint32_t c = 0; c < CA; ++c) {
+      uint64_t n = rows_of(c, CA);
       out.push_back(make("h1a", l, c, XEMA_KIND_CHUNK, XEMA_DTYPE_BF16, 2 * B * n * D, op.ln1a(c), op.kv(c) + 1));
       if (c == 0)
-        out.push_back(make("kv", l, -1, XEMA_KIND_FULL, XEMA_DTYPE_BF16, 2 * u, op.kv(0), op.attn(C - 1) + 1));
+        out.push_back(make("kv", l, -1, XEMA_KIND_FULL, XEMA_DTYPE_BF16, 2 * u, op.kv(0), op.attn(CB - 1) + 1));
     }
-    for (uint32_t c = 0; c < C; ++c) {
-      uint64_t n = (uint64_t)((int64_t)(c + 1) * S / C - (int64_t)c * S / C);
+    for (uint32_t c = 0; c < CB; ++c) {
+      uint64_t n = rows_of(c, CB);
       out.push_back(make("h1b", l, c, XEMA_KIND_CHUNK, XEMA_DTYPE_BF16, 2 * B * n * D, op.ln1b(c), op.q(c) + 1));
       out.push_back(make("q", l, c, XEMA_KIND_CHUNK, XEMA_DTYPE_BF16, 2 * B * n * D, op.q(c), op.attn(c) + 1));
       out.push_back(make("o", l, c, XEMA_KIND_CHUNK, XEMA_DTYPE_BF16, 2 * B * n * D, op.attn(c), op.proj(c) + 1));
       out.push_back(make("lse", l, c, XEMA_KIND_CHUNK, XEMA_DTYPE_F32, 4 * B * H * n, op.attn(c), op.attn(c) + 1));
       if (c == 0)
-        out.push_back(make("res", l, -1, XEMA_KIND_FULL, XEMA_DTYPE_F32, 2 * u, op.proj(0), op.ffn2(C - 1) + 1));
+        out.push_back(make("res", l, -1, XEMA_KIND_FULL, XEMA_DTYPE_F32, 2 * u, op.proj(0), op.ffn2(CC - 1) + 1));
     }
-    for (uint32_t c = 0; c < C; ++c) {
-      uint64_t n = (uint64_t)((int64_t)(c + 1) * S / C - (int64_t)c * S / C);
+    for (uint32_t c = 0; c < CC; ++c) {
+      uint64_t n = rows_of(c, CC);
       out.push_back(make("h2", l, c, XEMA_KIND_CHUNK, XEMA_DTYPE_BF16, 2 * B * n * D, op.ln2(c), op.ffn1(c) + 1));
       out.push_back(make("g", l, c, XEMA_KIND_CHUNK, XEMA_DTYPE_BF16, 2 * B * n * F, op.ffn1(c), op.ffn2(c) + 1));
       if (c == 0) {
         // the next hidden state: written chunk by chunk from FFN2_0 on; read by the next
         // block up to its last PROJ, or kept to the end if it is the output
         bool is_out = (l + 1 == L);
-        OpIndex nx{(l + 1) * ops_per_block, C};
-        uint32_t death = is_out ? total_ops : nx.proj(C - 1) + 1;
+        OpIndex nx{(l + 1) * ops_per_block, CA, CB, CC};
+        uint32_t death = is_out ? total_ops : nx.proj(CB - 1) + 1;
         out.push_back(make("hid", l + 1, -1, is_out ? XEMA_KIND_OUTPUT : XEMA_KIND_FULL, XEMA_DTYPE_BF16, u,
                            op.ffn2(0), death));
       }
@@ -223,6 +230,66 @@ int chunks_for_budget(const xema_config& cfg, uint64_t budget, int32_t max_chunk
   return XEMA_EBUDGET;
 }
 
+// Chunking only where the active-memory trace exceeds the budget: raise the chunk count of
+// exactly the phases that hold an over-budget op, one step at a time; if the laid-out peak still
+// exceeds the budget afterwards, raise the phase that holds the op with the most live bytes.
+int phase_chunks_for_budget(const xema_config& cfg, uint64_t budget, int32_t max_chunks, int32_t chunks[3],
+                            uint64_t* peak_out) {
+  int rc = validate_config(cfg);
+  if (rc) return rc;
+  if (max_chunks < 1) return XEMA_EINVAL;
+  const int32_t limit = (int32_t)std::min<int64_t>(max_chunks, seq_len(cfg));
+  int32_t c[3] = {1, 1, 1};
+  uint64_t smallest = ~uint64_t(0);
+  std::vector<xema_tensor> ts;
+  std::vector<uint64_t> offs, live;
+  while (true) {
+    uint32_t n_ops = 0;
+    rc = build_trace(cfg, c, ts, &n_ops);
+    if (rc) return rc;
+    offs.assign(ts.size(), 0);
+    uint64_t peak = 0;
+    rc = plan_arena(ts.data(), ts.size(), offs.data(), &peak, nullptr);
+    if (rc) return rc;
+    smallest = std::min(smallest, peak);
+    // active-memory trace by difference array
+    std::vector<int64_t> delta(n_ops + 1, 0);
+    for (const xema_tensor& t : ts) {
+      delta[t.birth] += (int64_t)t.bytes;
+      delta[t.death] -= (int64_t)t.bytes;
+    }
+    const uint32_t per_block = 1 + 3 * c[0] + 5 * c[1] + 3 * c[2];
+    auto phase_of = [&](uint32_t op) {
+      const uint32_t k = op % per_block;
+      return k < 1u + 3 * c[0] ? 0 : (k < 1u + 3 * c[0] + 5 * c[1] ? 1 : 2);
+    };
+    bool over[3] = {false, false, false};
+    int64_t cur = 0, best = -1;
+    uint32_t best_op = 0;
+    for (uint32_t op = 0; op < n_ops; ++op) {
+      cur += delta[op];
+      if ((uint64_t)cur > budget) over[phase_of(op)] = true;
+      if (cur > best) { best = cur; best_op = op; }
+    }
+    if (!over[0] && !over[1] && !over[2]) {
+      if (peak <= budget) {
+        for (int i = 0; i < 3; ++i) chunks[i] = c[i];
+        if (peak_out) *peak_out = peak;
+        return XEMA_OK;
+      }
+      over[phase_of(best_op)] = true;
+    }
+    for (int i = 0; i < 3; ++i) {
+      if (!over[i]) continue;
+      if (++c[i] > limit) {
+        chunks[0] = chunks[1] = chunks[2] = 0;
+        if (peak_out) *peak_out = smallest;
+        return XEMA_EBUDGET;
+      }
+    }
+  }
+}
+
 int rope_table(const xema_config& cfg, float* out) {
   int rc = validate_config(cfg);
   if (rc) return rc;
@@ -273,6 +340,26 @@ int xema_trace(const xema_config* cfg, int32_t chunks, xema_tensor* out, size_t 
   if (cap < ts.size() || !out) return XEMA_ENOSPC;
   std::memcpy(out, ts.data(), ts.size() * sizeof(xema_tensor));
   return XEMA_OK;
+}
+
+int xema_trace_phases(const xema_config* cfg, const int32_t chunks[3], xema_tensor* out, size_t cap,
+                      size_t* n_tensors, uint32_t* n_ops) {
+  if (!cfg || !chunks) return XEMA_EINVAL;
+  std::vector<xema_tensor> ts;
+  uint32_t ops = 0;
+  int rc = xema::build_trace(*cfg, chunks, ts, &ops);
+  if (rc) return rc;
+  if (n_tensors) *n_tensors = ts.size();
+  if (n_ops) *n_ops = ops;
+  if (cap < ts.size() || !out) return XEMA_ENOSPC;
+  std::memcpy(out, ts.data(), ts.size() * sizeof(xema_tensor));
+  return XEMA_OK;
+}
+
+int xema_phase_chunks_for_budget(const xema_config* cfg, uint64_t budget_bytes, int32_t max_chunks,
+                                 int32_t chunks[3], uint64_t* peak_bytes) {
+  if (!cfg || !chunks) return XEMA_EINVAL;
+  return xema::phase_chunks_for_budget(*cfg, budget_bytes, max_chunks, chunks, peak_bytes);
 }
 
 int xema_plan_arena(const xema_tensor* tensors, size_t n, uint64_t* offsets, uint64_t* peak_bytes,

@@ -106,7 +106,7 @@ using namespace xema;
 
 struct xema_plan {
   xema_config cfg;
-  int32_t chunks;
+  int32_t chunks[3];  // key/value, attention, feed-forward phase
   std::vector<xema_tensor> tensors;
   std::vector<uint64_t> offsets;
   std::unordered_map<std::string, size_t> index;
@@ -153,12 +153,17 @@ static int run_ops(const xema_plan* pl, size_t first, size_t n, void* stream) {
 extern "C" {
 
 int xema_plan_create(const xema_config* cfg, int32_t chunks, xema_plan** out) {
-  if (!cfg || !out) return XEMA_EINVAL;
+  const int32_t c3[3] = {chunks, chunks, chunks};
+  return xema_plan_create_phases(cfg, c3, out);
+}
+
+int xema_plan_create_phases(const xema_config* cfg, const int32_t chunks[3], xema_plan** out) {
+  if (!cfg || !out || !chunks) return XEMA_EINVAL;
   *out = nullptr;
   xema_plan* pl = new (std::nothrow) xema_plan();
   if (!pl) return XEMA_ENOSPC;
   pl->cfg = *cfg;
-  pl->chunks = chunks;
+  for (int i = 0; i < 3; ++i) pl->chunks[i] = chunks[i];
   pl->bound = false;
   pl->rope = nullptr;
   int rc = build_trace(*cfg, chunks, pl->tensors, &pl->n_ops);
@@ -184,7 +189,13 @@ int xema_plan_info(const xema_plan* plan, uint64_t* peak_bytes, uint64_t* max_li
   if (max_live_bytes) *max_live_bytes = plan->live;
   if (n_tensors) *n_tensors = plan->tensors.size();
   if (n_ops) *n_ops = plan->n_ops;
-  if (chunks) *chunks = plan->chunks;
+  if (chunks) *chunks = std::max(plan->chunks[0], std::max(plan->chunks[1], plan->chunks[2]));
+  return XEMA_OK;
+}
+
+int xema_plan_phase_chunks(const xema_plan* plan, int32_t chunks[3]) {
+  if (!plan || !chunks) return XEMA_EINVAL;
+  for (int i = 0; i < 3; ++i) chunks[i] = plan->chunks[i];
   return XEMA_OK;
 }
 
@@ -235,7 +246,7 @@ int xema_plan_bind(xema_plan* plan, void* arena_dev, uint64_t arena_bytes, const
   };
 
   const long long S = seq_len(c), D = c.hidden, F = c.ffn;
-  const int C = plan->chunks;
+  const int CA = plan->chunks[0], CB = plan->chunks[1], CC = plan->chunks[2];
   for (int l = 0; l < c.n_blocks; ++l) {
     const xema_block_weights& w = weights[l];
     const void* wp[12] = {w.w_mod, w.b_mod, w.w_qkv, w.b_qkv, w.g_q, w.g_k, w.w_o, w.b_o, w.w_1, w.b_1, w.w_2, w.b_2};
@@ -301,8 +312,8 @@ int xema_plan_bind(xema_plan* plan, void* arena_dev, uint64_t arena_bytes, const
     };
 
     // phase A: keys and values of every chunk
-    for (int ci = 0; ci < C; ++ci) {
-      const long long r0 = (long long)ci * S / C, r1 = (long long)(ci + 1) * S / C;
+    for (int ci = 0; ci < CA; ++ci) {
+      const long long r0 = (long long)ci * S / CA, r1 = (long long)(ci + 1) * S / CA;
       const int n = (int)(r1 - r0);
       uint8_t* h1a = at("h1a", l, ci);
       if (!h1a) return XEMA_EINVAL;
@@ -320,8 +331,8 @@ int xema_plan_bind(xema_plan* plan, void* arena_dev, uint64_t arena_bytes, const
       plan->ops.push_back(o);
     }
     // phase B: queries, attention and the gated output projection of every chunk
-    for (int ci = 0; ci < C; ++ci) {
-      const long long r0 = (long long)ci * S / C, r1 = (long long)(ci + 1) * S / C;
+    for (int ci = 0; ci < CB; ++ci) {
+      const long long r0 = (long long)ci * S / CB, r1 = (long long)(ci + 1) * S / CB;
       const int n = (int)(r1 - r0);
       uint8_t* h1b = at("h1b", l, ci);
       uint8_t* q = at("q", l, ci);
@@ -351,8 +362,8 @@ int xema_plan_bind(xema_plan* plan, void* arena_dev, uint64_t arena_bytes, const
       if (rc) return rc;
     }
     // phase C: feed-forward of every chunk
-    for (int ci = 0; ci < C; ++ci) {
-      const long long r0 = (long long)ci * S / C, r1 = (long long)(ci + 1) * S / C;
+    for (int ci = 0; ci < CC; ++ci) {
+      const long long r0 = (long long)ci * S / CC, r1 = (long long)(ci + 1) * S / CC;
       const int n = (int)(r1 - r0);
       uint8_t* h2 = at("h2", l, ci);
       uint8_t* g = at("g", l, ci);

@@ -22,12 +22,14 @@ class BlockSession:
     template: object with the xema_config field names (e.g. xema_inputs.Template).
     weights:  list (one per block) of dicts name -> uint16 bf16 bit patterns (numpy), or of
               dicts name -> torch tensors already on the device.
-    Either `chunks` or `budget_bytes` selects the chunk count.
+    Either `chunks` (one count, or a triple of per-phase counts) or `budget_bytes` selects
+    the chunking; with a budget, `per_phase` picks between the per-phase search (chunk only
+    the phases whose trace exceeds the budget) and one count for the whole block.
     """
 
-    def __init__(self, template, weights: Sequence[dict], chunks: Optional[int] = None,
+    def __init__(self, template, weights: Sequence[dict], chunks=None,
                  budget_bytes: Optional[int] = None, max_chunks: int = 64, device="cuda:0",
-                 arena: Optional[torch.Tensor] = None):
+                 arena: Optional[torch.Tensor] = None, per_phase: bool = True):
         if not torch.cuda.is_available():
             raise RuntimeError("a CUDA device is required (there is no CPU fallback)")
         self.device = torch.device(device)
@@ -37,12 +39,14 @@ class BlockSession:
         if chunks is None:
             if budget_bytes is None:
                 raise ValueError("give chunks or budget_bytes")
-            chunks, _ = xb.xema_chunks_for_budget(self.cfg, int(budget_bytes), max_chunks)
+            search = xb.xema_phase_chunks_for_budget if per_phase else xb.xema_chunks_for_budget
+            chunks, _ = search(self.cfg, int(budget_bytes), max_chunks)
             if chunks is None:
-                raise xb.XemaError(xb.XEMA_EBUDGET, "xema_chunks_for_budget")
+                raise xb.XemaError(xb.XEMA_EBUDGET, search.__name__)
         self.budget_bytes = budget_bytes
         self.plan = xb.Plan(self.cfg, chunks)
         self.chunks = chunks
+        self.phase_chunks = self.plan.phase_chunks
         if budget_bytes is not None and self.plan.peak_bytes > budget_bytes:
             raise xb.XemaError(xb.XEMA_EBUDGET, "plan peak exceeds the budget")
         if len(weights) != template.n_blocks:

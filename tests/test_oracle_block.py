@@ -175,7 +175,7 @@ def test_constant_v_and_zero_k(tiny):
 
 def test_chunked_equals_unchunked(tiny, tiny_out):
     t, W, x, temb = tiny
-    for C in (1, 2, 3, 5):
+    for C in (1, 2, 3, 5, (1, 1, 2), (2, 1, 3), (3, 2, 1)):
         out = ob.block_forward_chunked(t, W, x, temb, C)
         assert np.abs(out["y"] - tiny_out["y"]).max() < 1e-12
         assert np.abs(out["lse"] - tiny_out["lse"]).max() < 1e-12

@@ -221,3 +221,127 @@ def test_chunks_for_budget():
     assert arena.chunks_for_budget(template("flux", batch=4), 24 << 30, 8)[0] == 1
     assert arena.chunks_for_budget(template("longvideo"), 8 << 30, 8)[0] == 1
     assert arena.chunks_for_budget(template("longvideo"), 4 << 30, 8)[0] == 2
+
+
+# ---- per-phase chunk counts ("Applying Mitigation Only Where Needed") ---------------------
+
+def _closed_form_phase_live(t, counts):
+    """Largest live-byte sum inside each phase of a single block, written out per op from the
+    block's data flow (not from the recorder): which full-size tensors exist at that point
+    plus the chunk-sized ones of the largest chunk."""
+    A = trace.align_up
+    B, S, D, H, F = t.batch, t.seq, t.hidden, t.heads, t.ffn
+    ca, cb, cc = counts
+    u, mod, kv, res = A(2 * B * S * D), A(24 * B * D), A(4 * B * S * D), A(4 * B * S * D)
+    big = lambda C: -(-S // C)
+    ck = lambda n, w: A(2 * B * n * w)
+    # phase A peaks at a KV op: block input, modulation, the K/V tensor, the LN output chunk
+    pa = max(A(2 * B * t.temb_dim) + u + mod, u + mod + kv + ck(big(ca), D))
+    # phase B: ATTN holds q, o and lse of the chunk; res exists from the first PROJ on
+    n = big(cb)
+    attn = u + mod + kv + 2 * ck(n, D) + A(4 * B * H * n)
+    if cb == 1:
+        pb = max(attn, u + mod + ck(n, D) + res)
+    else:
+        pb = attn + res
+    # phase C: FFN1 holds the LN output and the GELU output of the chunk; the next hidden
+    # state exists from the first FFN2 on
+    n = big(cc)
+    if cc == 1:
+        pc = mod + res + max(ck(n, D) + ck(n, F), ck(n, F) + u)
+    else:
+        pc = mod + res + u + ck(n, D) + ck(n, F)
+    return pa, pb, pc
+
+
+@pytest.mark.parametrize("name", ["tiny", "cogvideox", "flux", "longvideo"])
+def test_phase_trace_closed_form(name):
+    t = template(name)
+    for counts in [(1, 1, 1), (1, 1, 2), (1, 1, 3), (2, 1, 1), (1, 2, 1), (3, 2, 5), (4, 4, 4), (2, 7, 3)]:
+        ts, n_ops = trace.trace(t, counts)
+        assert n_ops == 1 + 3 * counts[0] + 5 * counts[1] + 3 * counts[2]
+        live = arena.live_per_op(ts, n_ops)
+        got = [0, 0, 0]
+        for op, b in enumerate(live):
+            ph = arena.phase_of_op(t, counts, op)
+            got[ph] = max(got[ph], b)
+        assert tuple(got) == _closed_form_phase_live(t, counts), (name, counts)
+        assert max(got) == arena.max_live_bytes(ts, n_ops)
+
+
+def test_phase_trace_reduces_to_uniform():
+    for name in ("tiny", "step"):
+        t = template(name)
+        for C in (1, 2, 3):
+            assert trace.trace(t, (C, C, C)) == trace.trace(t, C)
+
+
+def test_phase_trace_lifetimes_tiny():
+    """(C_A, C_B, C_C) = (2, 1, 3) on the tiny template, op by op:
+    0 MOD | 1 LN1A_0 2 KV_0 3 KROPE_0 4 LN1A_1 5 KV_1 6 KROPE_1 | 7 LN1B 8 Q 9 QROPE 10 ATTN
+    11 PROJ | 12 LN2_0 13 FFN1_0 14 FFN2_0 15 LN2_1 16 FFN1_1 17 FFN2_1 18 LN2_2 19 FFN1_2
+    20 FFN2_2."""
+    t = template("tiny")
+    ts, n_ops = trace.trace(t, (2, 1, 3))
+    assert n_ops == 21
+    life = {d["name"]: (d["birth"], d["death"]) for d in ts}
+    assert life == {
+        "temb": (0, 1), "hid0": (0, 12), "mod0": (0, 21),
+        "h1a0_0": (1, 3), "kv0": (2, 11), "h1a0_1": (4, 6),
+        "h1b0_0": (7, 9), "q0_0": (8, 11), "o0_0": (10, 12), "lse0_0": (10, 11), "res0": (11, 21),
+        "h20_0": (12, 14), "g0_0": (13, 15), "hid1": (14, 21),
+        "h20_1": (15, 17), "g0_1": (16, 18), "h20_2": (18, 20), "g0_2": (19, 21),
+    }
+    S = t.seq
+    rows = {d["name"]: d["bytes"] for d in ts}
+    assert rows["h1a0_0"] == trace.align_up(2 * t.batch * (S // 2) * t.hidden)
+    assert rows["g0_1"] == trace.align_up(2 * t.batch * (2 * S // 3 - S // 3) * t.ffn)
+
+
+@pytest.mark.parametrize("name", ["tiny", "cogvideox"])
+def test_phase_plan_valid_and_tight(name):
+    t = template(name)
+    for counts in itertools.product((1, 2, 3), repeat=3):
+        ts, n_ops = trace.trace(t, counts)
+        offsets, peak = arena.plan_arena(ts)
+        assert arena.overlapping_pairs(ts, offsets) == []
+        assert peak == arena.max_live_bytes(ts, n_ops)
+
+
+@pytest.mark.parametrize("name", ["tiny", "cogvideox", "flux"])
+def test_phase_chunks_for_budget_is_minimal(name):
+    """The search result fits, and no triple with a smaller total chunk count does (brute
+    force over all triples up to 4 per phase)."""
+    t = template(name)
+    peaks = {c: arena.plan_arena(trace.trace(t, c)[0])[1] for c in itertools.product((1, 2, 3, 4), repeat=3)}
+    p1 = peaks[(1, 1, 1)]
+    for frac in (1.0, 0.95, 0.85, 0.79, 0.75, 0.73):
+        budget = int(p1 * frac)
+        counts, peak = arena.phase_chunks_for_budget(t, budget, 4)
+        feasible = [c for c, p in peaks.items() if p <= budget]
+        assert counts is not None and peak == peaks[counts] and peak <= budget
+        assert sum(counts) == min(sum(c) for c in feasible), (name, frac, counts)
+    # chunking the attention phase never helps: its floor is the unchunked attention peak
+    assert min(peaks[(a, b, c)] for a, b, c in peaks if b > 1) > min(peaks.values())
+
+
+def test_phase_chunks_for_budget_values():
+    t = template("cogvideox")
+    MiB = 1 << 20
+    assert arena.phase_chunks_for_budget(t, 768 * MiB, 16) == ((1, 1, 1), 764583936)
+    # 640 MiB: one count for the whole block needs C = 2 and reserves 657 074 688 bytes;
+    # chunking the feed-forward phase alone reserves less with 3 fewer launches
+    assert arena.chunks_for_budget(t, 640 * MiB, 16) == (2, 657074688)
+    assert arena.phase_chunks_for_budget(t, 640 * MiB, 16) == ((1, 1, 2), 600760320)
+    assert arena.phase_chunks_for_budget(t, 576 * MiB, 16) == ((1, 1, 2), 600760320)
+    assert arena.phase_chunks_for_budget(t, 560 * MiB, 16) == ((1, 1, 3), 549565440)
+    # 525 MiB is below every uniform plan up to 16 chunks but (1, 1, 3) fits
+    assert arena.chunks_for_budget(t, 525 * MiB, 16)[0] is None
+    assert arena.phase_chunks_for_budget(t, 525 * MiB, 16) == ((1, 1, 3), 549565440)
+    # the floor: block input, K/V, q, o and lse of the unchunked attention
+    assert arena.phase_chunks_for_budget(t, 549565440 - 1, 16)[0] is None
+    # non-binding budgets stay unchunked
+    assert arena.phase_chunks_for_budget(template("longvideo"), 8 << 30, 8)[0] == (1, 1, 1)
+    assert arena.phase_chunks_for_budget(template("longvideo"), 4 << 30, 8)[0] == (1, 1, 2)
+    # the 42-block step: same counts as one block (the budget binds inside a block)
+    assert arena.phase_chunks_for_budget(template("step"), 640 * MiB, 16)[0] == (1, 1, 2)

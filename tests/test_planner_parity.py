@@ -93,3 +93,69 @@ def test_rope_table_against_oracle_angles():
         assert np.array_equal(tab[..., 1], np.sin(ang).astype(np.float32))
     # text tokens are left unrotated
     assert np.all(tab[:t.s_text, :, 0] == 1.0) and np.all(tab[:t.s_text, :, 1] == 0.0)
+
+
+# ---- per-phase chunk counts ---------------------------------------------------------------
+
+PHASE_TRIPLES = [(1, 1, 1), (1, 1, 2), (1, 1, 3), (2, 1, 3), (3, 2, 1), (1, 4, 2), (5, 3, 7), (16, 1, 9)]
+
+
+@pytest.mark.parametrize("name,batch", CASES + [("step", 1)])
+def test_phase_trace_offsets_peak_bit_exact(name, batch):
+    t = template(name, batch=batch)
+    cfg = xb.make_config(t)
+    for counts in PHASE_TRIPLES if name != "step" else PHASE_TRIPLES[:4]:
+        want, want_ops = o_trace.trace(t, counts)
+        got, got_ops = xb.xema_trace_phases(cfg, counts)
+        assert got_ops == want_ops and got == want, (name, counts)
+        offs, peak, live = xb.xema_plan_arena(got)
+        w_offs, w_peak = o_arena.plan_arena(want)
+        assert offs == w_offs and peak == w_peak
+        plan = xb.Plan(cfg, counts)
+        assert plan.phase_chunks == counts and plan.chunks == max(counts)
+        assert plan.peak_bytes == w_peak and plan.n_ops == want_ops
+        assert [d["offset"] for d in plan.tensors()] == w_offs
+        plan.close()
+
+
+def test_phase_trace_uniform_equals_trace():
+    t = template("cogvideox")
+    cfg = xb.make_config(t)
+    for C in (1, 2, 5):
+        assert xb.xema_trace_phases(cfg, (C, C, C)) == xb.xema_trace(cfg, C)
+        a, b = xb.Plan(cfg, C), xb.Plan(cfg, (C, C, C))
+        assert (a.peak_bytes, a.n_ops, a.phase_chunks) == (b.peak_bytes, b.n_ops, b.phase_chunks)
+
+
+def test_phase_trace_rejects_bad_counts():
+    t = template("tiny")
+    cfg = xb.make_config(t)
+    for bad in [(0, 1, 1), (1, -1, 1), (1, 1, t.seq + 1)]:
+        with pytest.raises(xb.XemaError) as e:
+            xb.xema_trace_phases(cfg, bad)
+        assert e.value.status == xb.XEMA_EINVAL
+        with pytest.raises(xb.XemaError):
+            xb.Plan(cfg, bad)
+    got, n_ops = xb.xema_trace_phases(cfg, (t.seq, 1, t.seq))
+    assert n_ops == 1 + 3 * t.seq + 5 + 3 * t.seq
+
+
+def test_phase_chunks_for_budget_bit_exact():
+    GiB = 1 << 30
+    sweeps = [
+        ("cogvideox", 1, [764583936, 764583935, 657074688, 600760320, 600760319, 549565440, 549565439,
+                          525 << 20, 1 << 40, 1]),
+        ("flux", 1, [24 * GiB, 150 << 20, 142073856, 142073855]), ("flux", 4, [24 * GiB, 700 << 20]),
+        ("longvideo", 1, [8 * GiB, 4 * GiB, int(3.5 * GiB), int(3.25 * GiB), 3 * GiB]),
+        ("longvideo", 2, [8 * GiB, 16 * GiB]),
+        ("step", 1, [768 << 20, 640 << 20, 576 << 20]),
+        ("tiny", 1, [2076672, 1786368, 1634304, 1634303, 1496064, 1496063]),
+    ]
+    for name, batch, budgets in sweeps:
+        t = template(name, batch=batch)
+        cfg = xb.make_config(t)
+        for budget in budgets:
+            got = xb.xema_phase_chunks_for_budget(cfg, budget, 16)
+            assert got == o_arena.phase_chunks_for_budget(t, budget, 16), (name, budget)
+    with pytest.raises(xb.XemaError):
+        xb.xema_phase_chunks_for_budget(xb.make_config(template("tiny")), 1 << 30, 0)
