@@ -6,7 +6,8 @@
 
 One step = one pass of the whole hot path (modulation, LayerNorm+modulate, QKV GEMMs, RMSNorm +
 RoPE, attention, gated projection, FFN) over one batch of seeded synthetic input, sequence-
-chunked with the smallest chunk count whose arena peak fits the byte budget.  Prints ONE JSON
+chunked only in the phases whose memory trace exceeds the byte budget (per-phase chunk counts;
+--uniform-chunks uses one count for the whole block instead).  Prints ONE JSON
 line (see the keys below).  Under torchrun every rank runs the same workload on its own GPU
 (independent replicas, no data-path collective); the value is the sum over ranks divided by the
 slowest rank's time.
@@ -188,8 +189,11 @@ def main():
     ap.add_argument("--impl", default="xema", choices=["xema", "reference"])
     ap.add_argument("--workload", default="cogvideox", choices=["tiny", "cogvideox", "flux", "longvideo", "step"])
     ap.add_argument("--budget-mib", type=float, default=640.0,
-                    help="activation byte budget; the smallest chunk count whose arena peak fits is used")
-    ap.add_argument("--chunks", type=int, default=0, help="force a chunk count instead of a budget")
+                    help="activation byte budget; the least chunking whose arena peak fits is used")
+    ap.add_argument("--chunks", default="", help="force a chunk count C, or per-phase counts CA,CB,CC, "
+                                                 "instead of a budget")
+    ap.add_argument("--uniform-chunks", action="store_true",
+                    help="budget search over one chunk count for all three phases")
     ap.add_argument("--cpu-rows", type=int, default=CPU_SAMPLE_ROWS)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep", action="store_true", help="also time chunk counts 1, 2, 4, 8 (outside the timed region)")
@@ -217,10 +221,15 @@ def main():
 
     t = template(args.workload)
     cfg = xb.make_config(t)
-    budget = None if args.chunks else int(args.budget_mib * (1 << 20))
+    forced = None
+    if args.chunks:
+        c = [int(v) for v in args.chunks.split(",")]
+        forced = c[0] if len(c) == 1 else tuple(c)
+    budget = None if forced else int(args.budget_mib * (1 << 20))
     weights = [make_block_weights(t, l) for l in range(t.n_blocks)]
     x_bits, temb_bits = make_activations(t)
-    sess = BlockSession(t, weights, chunks=args.chunks or None, budget_bytes=budget, device=dev)
+    sess = BlockSession(t, weights, chunks=forced, budget_bytes=budget, device=dev,
+                        per_phase=not args.uniform_chunks)
     n_launch = sess.plan.n_ops            # logical ops of the trace (fused ones launch nothing)
     n_kernels = sess.plan.launch_count()  # kernels actually launched per step
     ops = [sess.plan.op(i) for i in range(n_launch)]
@@ -288,7 +297,7 @@ def main():
     if args.sweep and rank == 0:
         sweep = {}
         dev_w = sess.weights
-        for C in (1, 2, 4, 8):
+        for C in (1, 2, 4, 8, (1, 1, 2), (1, 1, 3)):
             s2 = BlockSession(t, dev_w, chunks=C, device=dev)
             s2.set_inputs(x_bits, temb_bits)
             for _ in range(3):
@@ -301,7 +310,7 @@ def main():
             b.record(stream)
             torch.cuda.synchronize(dev)
             ms = a.elapsed_time(b) / 10
-            sweep[str(C)] = {"ms": ms, "tflops": flops / ms / 1e9, "arena_bytes": s2.plan.peak_bytes}
+            sweep[str(C).replace(" ", "")] = {"ms": ms, "tflops": flops / ms / 1e9, "arena_bytes": s2.plan.peak_bytes}
             del s2
             torch.cuda.empty_cache()
 
@@ -350,7 +359,9 @@ def main():
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": args.workload, "batch": t.batch, "tokens": t.seq, "hidden": t.hidden,
                    "heads": t.heads, "head_dim": t.head_dim, "ffn": t.ffn, "n_blocks": t.n_blocks,
-                   "budget_bytes": budget, "chunks": sess.chunks, "arena_bytes": sess.plan.peak_bytes,
+                   "budget_bytes": budget, "chunks": list(sess.phase_chunks),
+                   "chunk_search": "forced" if forced else ("uniform" if args.uniform_chunks else "per_phase"),
+                   "arena_bytes": sess.plan.peak_bytes,
                    "trace_max_live_bytes": sess.plan.max_live_bytes,
                    "device_bytes_allocated_by_forward": int(free_before - free_after),
                    "l2": "inputs larger than L2 (weights 245 MB + arena per block)",

@@ -123,11 +123,33 @@ def test_forward_stays_inside_the_planned_arena(tiny_case):
 def test_budget_selects_chunks_and_fits(tiny_case):
     t, w, x, temb, ref = tiny_case
     for budget, want in ((2076672, 1), (2076671, 2), (1786368, 2), (1700000, 3)):
-        s = BlockSession(t, [w], budget_bytes=budget)
+        s = BlockSession(t, [w], budget_bytes=budget, per_phase=False)
         assert s.chunks == want and s.plan.peak_bytes <= budget and s.arena.numel() == s.plan.peak_bytes
     s.set_inputs(x, temb)
     s.forward()
     assert_close(bits_to_f64(s.output_bits()), ref["y"], "budgeted tiny block")
+
+
+def test_per_phase_chunks_are_bit_identical_and_fit(tiny_case):
+    """Chunking only the phases that need it: any triple of per-phase counts gives the bits of
+    the unchunked block; the budget search picks (1, 1, C) and its plan fits the budget."""
+    t, w, x, temb, ref = tiny_case
+    _, base = _run(t, [w], x, temb, 1)
+    for counts in [(1, 1, 2), (1, 1, 3), (2, 1, 3), (3, 2, 1), (1, 4, 2), (5, 3, 7)]:
+        s, y = _run(t, [w], x, temb, counts)
+        assert s.phase_chunks == counts and s.plan.n_ops == 1 + 3 * counts[0] + 5 * counts[1] + 3 * counts[2]
+        assert np.array_equal(y, base), counts
+    for budget, want in ((2076672, (1, 1, 1)), (2076671, (1, 1, 2)), (1634304, (1, 1, 2)), (1634303, (1, 1, 3)),
+                         (1496064, (1, 1, 3))):
+        s = BlockSession(t, [w], budget_bytes=budget)
+        assert s.chunks == want and s.plan.peak_bytes <= budget and s.arena.numel() == s.plan.peak_bytes
+        s.set_inputs(x, temb)
+        s.forward()
+        assert np.array_equal(s.output_bits(), base), budget
+    assert_close(bits_to_f64(base), ref["y"], "per-phase tiny block")
+    with pytest.raises(xb.XemaError) as e:
+        BlockSession(t, [w], budget_bytes=1496063)
+    assert e.value.status == xb.XEMA_EBUDGET
 
 
 def test_batch_two_small_block():
@@ -195,7 +217,7 @@ def test_full_size_block_sampled_rows(name):
     first = None
     for C in (1, 2, 4, 8):
         peak = xb.Plan(cfg, C).peak_bytes
-        s = BlockSession(t, [dev_w or w], budget_bytes=peak)
+        s = BlockSession(t, [dev_w or w], budget_bytes=peak, per_phase=False)
         dev_w = s.weights[0]
         assert s.chunks == C and s.arena.numel() == peak
         s.set_inputs(x, temb)
@@ -217,6 +239,15 @@ def test_full_size_block_sampled_rows(name):
             assert st["cos"] >= 0.9995
         else:
             assert np.array_equal(first, y), C
+        del s
+        torch.cuda.empty_cache()
+    # per-phase search at the budgets the uniform search needs C = 2 and C >= 6 for
+    for budget, want, peak in ((640 << 20, (1, 1, 2), 600760320), (560 << 20, (1, 1, 3), 549565440)):
+        s = BlockSession(t, [dev_w], budget_bytes=budget)
+        assert s.chunks == want and s.arena.numel() == peak
+        s.set_inputs(x, temb)
+        s.forward()
+        assert np.array_equal(first, s.output_bits()), want
         del s
         torch.cuda.empty_cache()
 

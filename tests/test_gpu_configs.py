@@ -42,7 +42,7 @@ def test_flux_block_under_24gib(batch):
     w = make_block_weights(t, 0)
     x, temb = make_activations(t)
     s = BlockSession(t, [w], budget_bytes=24 * GiB)
-    assert s.chunks == 1                       # the budget is not binding for this template
+    assert s.phase_chunks == (1, 1, 1)         # the budget is not binding for this template
     assert s.plan.peak_bytes == s.plan.max_live_bytes <= 24 * GiB
     s.set_inputs(x, temb)
     s.forward()
@@ -67,7 +67,7 @@ def test_longvideo_block_binding_budget():
     assert xb.xema_chunks_for_budget(cfg, int(3.5 * GiB), 16)[0] == 3
     w = make_block_weights(t, 0)
     x, temb = make_activations(t)
-    s = BlockSession(t, [w], budget_bytes=4 * GiB)
+    s = BlockSession(t, [w], budget_bytes=4 * GiB, per_phase=False)
     assert s.chunks == 2 and s.plan.peak_bytes <= 4 * GiB and s.arena.numel() == s.plan.peak_bytes
     s.set_inputs(x, temb)
     s.forward()
@@ -84,8 +84,10 @@ def test_cogvideox_step_42_blocks_teacher_forced():
     t = template("step")
     cfg = xb.make_config(t)
     budget = 640 << 20
-    C, peak = xb.xema_chunks_for_budget(cfg, budget, 16)
-    assert C == 2 and peak == 657075712
+    C, peak_uniform = xb.xema_chunks_for_budget(cfg, budget, 16)
+    assert C == 2 and peak_uniform == 657075712
+    counts, peak = xb.xema_phase_chunks_for_budget(cfg, budget, 16)
+    assert counts == (1, 1, 2) and peak == 600761344
     weights = []
     keep = {}
     for l in range(t.n_blocks):
