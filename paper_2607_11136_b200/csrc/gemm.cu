@@ -13,6 +13,9 @@
 //             other accumulator
 // A row's result depends only on (row, N, K): the K loop always runs in the same order and the
 // tile shape is chosen from N alone, so outputs are bit-identical however rows are chunked.
+#include <cstdio>
+#include <cstdlib>
+
 #include "kernels.h"
 #include "sm100.cuh"
 
@@ -166,6 +169,38 @@ __device__ __forceinline__ void epilogue_head_norm_rope(const GemmParams& p, int
   }
 }
 
+// The finished BN-wide accumulator row of one thread (TMEM address t_addr) -> global memory.
+template <int BN, int EPI>
+__device__ __forceinline__ void epilogue_row(const GemmParams& p, int b, int row, int n_base, uint32_t t_addr) {
+  if constexpr (EPI == XEMA_EPI_BIAS_NORM_ROPE) {
+    // head by head; heads at or beyond norm_cols (the V half of a KV product) get the bias only
+#pragma unroll 1
+    for (int hc = 0; hc < BN; hc += p.head_dim) {
+      const int n0 = n_base + hc;
+      if (n0 < p.norm_cols) {
+        if (p.head_dim == 64) epilogue_head_norm_rope<64>(p, b, row, n0, t_addr + hc);
+        else epilogue_head_norm_rope<128>(p, b, row, n0, t_addr + hc);
+      } else {
+#pragma unroll 1
+        for (int ch = 0; ch < p.head_dim / 32; ++ch) {
+          uint32_t r[32];
+          tmem_ld32(t_addr + hc + ch * 32, r);
+          tmem_ld_wait();
+          epilogue_chunk<XEMA_EPI_BIAS>(p, b, row, n0 + ch * 32, r);
+        }
+      }
+    }
+  } else {
+#pragma unroll 1
+    for (int ch = 0; ch < BN / 32; ++ch) {
+      uint32_t r[32];
+      tmem_ld32(t_addr + ch * 32, r);
+      tmem_ld_wait();
+      epilogue_chunk<EPI>(p, b, row, n_base + ch * 32, r);
+    }
+  }
+}
+
 struct TileCoord {
   int b, mt, nt;
 };
@@ -259,39 +294,47 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     }
   } else if (warp == 1) {
     // ---------------- MMA issuer ----------------
-    if (lane == 0) {
+    // The whole warp walks the loop and waits together; one elected lane issues.  (A lone
+    // thread of a diverged warp issues MMAs markedly slower than the tensor pipe retires them.)
+    {
       constexpr uint32_t idesc = idesc_bf16_f32(BM, BN, false, false);
-      // The issuing thread is a lone dependent instruction stream, so its loop is kept short:
-      // descriptors are built once and advanced by adding constants (the start-address field
+      // Descriptors are built once and advanced by adding constants (the start-address field
       // counts 16-byte units and never carries out of its 14 bits inside shared memory).
       const uint64_t a_desc0 = smem_desc_sw128(smem_u32(smem), 16, 1024);
       const uint64_t b_desc0 = smem_desc_sw128(smem_u32(smem + A_TILE_BYTES), 16, 1024);
+      auto wait_all = [&](uint64_t* bar, uint32_t parity) -> bool {
+        return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
+      };
       int stage = 0;
       uint32_t phase = 0;
       int acc = 0;
       uint32_t acc_phase = 0;
       bool ok = true;
       for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
-        if (!(ok = mbar_wait(&tmem_empty[acc], acc_phase ^ 1, abort_flag))) break;
+        if (!(ok = wait_all(&tmem_empty[acc], acc_phase ^ 1))) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * BN;
         uint32_t accumulate = 0;
 #pragma unroll 1
         for (int kb = 0; kb < k_blocks; ++kb) {
-          if (!(ok = mbar_wait(&full[stage], phase, abort_flag))) break;
+          if (!(ok = wait_all(&full[stage], phase))) break;
           tc_fence_after();
-          const uint64_t soff = (uint64_t)(stage * (Cfg::STAGE_BYTES >> 4));
-          const uint64_t da = a_desc0 + soff, db = b_desc0 + soff;
-          mma_ss(d_tmem, da, db, idesc, accumulate);
-          mma_ss(d_tmem, da + 2, db + 2, idesc, 1);
-          mma_ss(d_tmem, da + 4, db + 4, idesc, 1);
-          mma_ss(d_tmem, da + 6, db + 6, idesc, 1);
-          mma_commit(&empty[stage]);
+          if (elect_one()) {
+            const uint64_t soff = (uint64_t)(stage * (Cfg::STAGE_BYTES >> 4));
+            const uint64_t da = a_desc0 + soff, db = b_desc0 + soff;
+            mma_ss(d_tmem, da, db, idesc, accumulate);
+            mma_ss(d_tmem, da + 2, db + 2, idesc, 1);
+            mma_ss(d_tmem, da + 4, db + 4, idesc, 1);
+            mma_ss(d_tmem, da + 6, db + 6, idesc, 1);
+            mma_commit(&empty[stage]);
+          }
+          __syncwarp();
           accumulate = 1;
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
         if (!ok) break;
-        mma_commit(&tmem_full[acc]);
+        if (elect_one()) mma_commit(&tmem_full[acc]);
+        __syncwarp();
         if (++acc == 2) { acc = 0; acc_phase ^= 1; }
       }
     }
@@ -309,33 +352,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
       tc_fence_after();
       const int row = c.mt * BM + quad * 32 + lane;
       const uint32_t t_addr = tmem_base + ((uint32_t)(quad * 32) << 16) + acc * BN;
-      if constexpr (EPI == XEMA_EPI_BIAS_NORM_ROPE) {
-        // head by head; heads at or beyond norm_cols (the V half of a KV product) get the bias only
-#pragma unroll 1
-        for (int hc = 0; hc < BN; hc += p.head_dim) {
-          const int n0 = c.nt * BN + hc;
-          if (n0 < p.norm_cols) {
-            if (p.head_dim == 64) epilogue_head_norm_rope<64>(p, c.b, row, n0, t_addr + hc);
-            else epilogue_head_norm_rope<128>(p, c.b, row, n0, t_addr + hc);
-          } else {
-#pragma unroll 1
-            for (int ch = 0; ch < p.head_dim / 32; ++ch) {
-              uint32_t r[32];
-              tmem_ld32(t_addr + hc + ch * 32, r);
-              tmem_ld_wait();
-              epilogue_chunk<XEMA_EPI_BIAS>(p, c.b, row, n0 + ch * 32, r);
-            }
-          }
-        }
-      } else {
-#pragma unroll 1
-        for (int ch = 0; ch < BN / 32; ++ch) {
-          uint32_t r[32];
-          tmem_ld32(t_addr + ch * 32, r);
-          tmem_ld_wait();
-          epilogue_chunk<EPI>(p, c.b, row, c.nt * BN + ch * 32, r);
-        }
-      }
+      epilogue_row<BN, EPI>(p, c.b, row, c.nt * BN, t_addr);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&tmem_empty[acc]);
@@ -348,6 +365,174 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_base, Cfg::TMEM_COLS);
+  }
+  if (threadIdx.x == 0 && *abort_flag && p.status) atomicExch(p.status, STATUS_TIMEOUT_MBARRIER);
+}
+
+
+// ---------------------------------------------------------------------------------------------
+// CTA-pair variant (N a multiple of 256): two CTAs on neighbouring SMs share one 256 x 256
+// output tile.  Each CTA loads its own 128 rows of A and one half (128 rows) of the W tile, so a
+// stage costs 32 KB of shared-memory fill per SM instead of 48 KB and every MMA reads 8 KB of
+// operands per SM instead of 12 KB; the even CTA issues tcgen05.mma.cta_group::2 (M = 256),
+// which accumulates 128 rows x 256 columns in the TMEM of each CTA.
+//   full[s]        barrier of the even CTA: its producer expects the bytes of both CTAs, and
+//                  both CTAs' loads complete on it (an expect-tx arrival sent from the peer
+//                  CTA for every stage halved the speed of the whole loop)
+//   empty[s]       one barrier per CTA, released for both by a multicast commit
+//   tmem_full[a]   one barrier per CTA, same commit form
+//   tmem_empty[a]  barrier of the even CTA: the four epilogue warps of both CTAs arrive
+// The K loop and the per-instruction summation are the same for every row, so results do not
+// depend on how rows are chunked.
+constexpr int PAIR_BN = 256;
+constexpr int PAIR_STAGES = 6;
+constexpr int PAIR_B_HALF_BYTES = (PAIR_BN / 2) * BK * 2;
+constexpr int PAIR_STAGE_BYTES = A_TILE_BYTES + PAIR_B_HALF_BYTES;
+constexpr int PAIR_SMEM_BYTES = 1024 + PAIR_STAGES * PAIR_STAGE_BYTES + 256;
+constexpr int PAIR_TMEM_COLS = 2 * PAIR_BN;
+
+template <int EPI>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
+gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w,
+                      const GemmParams p) {
+  constexpr int STAGES = PAIR_STAGES;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* bar_base = smem + STAGES * PAIR_STAGE_BYTES;
+  uint64_t* full = reinterpret_cast<uint64_t*>(bar_base);
+  uint64_t* empty = full + STAGES;
+  uint64_t* tmem_full = empty + STAGES;
+  uint64_t* tmem_empty = tmem_full + 2;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tmem_empty + 2);
+  volatile uint32_t* abort_flag = tmem_slot + 1;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();            // 0: even CTA (issues the MMAs), 1: its peer
+  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+  const int m_tiles = (p.rows + 2 * BM - 1) / (2 * BM);   // tiles of 256 rows
+  const int n_tiles = p.N / PAIR_BN;
+  const int k_blocks = p.K / BK;
+  const int total_tiles = p.batch * m_tiles * n_tiles;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(&full[s], 1);
+      mbar_init(&empty[s], 1);
+    }
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(&tmem_full[s], 1);
+      mbar_init(&tmem_empty[s], 8);
+    }
+    *abort_flag = 0;
+    fence_mbar_init();
+    prefetch_tmap(&map_a);
+    prefetch_tmap(&map_w);
+  }
+  if (warp == 1) {
+    tmem_alloc_pair(tmem_slot, PAIR_TMEM_COLS);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_arrive();      // both CTAs' barriers exist before anything arrives on them remotely
+  cluster_wait();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ---------------- TMA producer (one per CTA) ----------------
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = pair; ok && tile < total_tiles; tile += n_pairs) {
+        const TileCoord c = tile_coord(tile, m_tiles, n_tiles);
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          if (!(ok = mbar_wait(&empty[stage], phase ^ 1, abort_flag))) break;
+          uint8_t* sa = smem + stage * PAIR_STAGE_BYTES;
+          uint8_t* sb = sa + A_TILE_BYTES;
+          const uint32_t full0 = mapa_shared(smem_u32(&full[stage]), 0);
+          if (rank == 0) mbar_expect_tx(&full[stage], 2 * PAIR_STAGE_BYTES);
+          tma_load_3d_pair(sa, &map_a, full0, kb * BK, (c.mt * 2 + (int)rank) * BM, c.b);
+          tma_load_3d_pair(sb, &map_w, full0, kb * BK, c.nt * PAIR_BN + (int)rank * (PAIR_BN / 2), 0);
+          if (++stage == STAGES) { stage = 0; phase ^= 1; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer (even CTA only; converged warp, one elected lane) ----------------
+    if (rank == 0) {
+      constexpr uint32_t idesc = idesc_bf16_f32(2 * BM, PAIR_BN, false, false);
+      const uint64_t a_desc0 = smem_desc_sw128(smem_u32(smem), 16, 1024);
+      const uint64_t b_desc0 = smem_desc_sw128(smem_u32(smem + A_TILE_BYTES), 16, 1024);
+      auto wait_all = [&](uint64_t* bar, uint32_t parity) -> bool {
+        return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
+      };
+      int stage = 0;
+      uint32_t phase = 0;
+      int acc = 0;
+      uint32_t acc_phase = 0;
+      bool ok = true;
+      for (int tile = pair; ok && tile < total_tiles; tile += n_pairs) {
+        // the peer's epilogue warps arrive on this barrier from their own CTA: cluster-scope acquire
+        if (!(ok = __all_sync(0xffffffffu, mbar_wait_cluster(&tmem_empty[acc], acc_phase ^ 1, abort_flag)))) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * PAIR_BN;
+        uint32_t accumulate = 0;
+#pragma unroll 1
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          if (!(ok = wait_all(&full[stage], phase))) break;
+          tc_fence_after();
+          if (elect_one()) {
+            const uint64_t soff = (uint64_t)(stage * (PAIR_STAGE_BYTES >> 4));
+            const uint64_t da = a_desc0 + soff, db = b_desc0 + soff;
+            mma_ss_pair(d_tmem, da, db, idesc, accumulate);
+            mma_ss_pair(d_tmem, da + 2, db + 2, idesc, 1);
+            mma_ss_pair(d_tmem, da + 4, db + 4, idesc, 1);
+            mma_ss_pair(d_tmem, da + 6, db + 6, idesc, 1);
+            mma_commit_pair(&empty[stage]);
+          }
+          __syncwarp();
+          accumulate = 1;
+          if (++stage == STAGES) { stage = 0; phase ^= 1; }
+        }
+        if (!ok) break;
+        if (elect_one()) mma_commit_pair(&tmem_full[acc]);
+        __syncwarp();
+        if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+      }
+    }
+  } else {
+    // ---------------- epilogue (both CTAs, each its own 128 rows) ----------------
+    const int quad = warp & 3;
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    bool ok = true;
+    for (int tile = pair; ok && tile < total_tiles; tile += n_pairs) {
+      const TileCoord c = tile_coord(tile, m_tiles, n_tiles);
+      ok = mbar_wait(&tmem_full[acc], acc_phase, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      const int row = (c.mt * 2 + (int)rank) * BM + quad * 32 + lane;
+      const uint32_t t_addr = tmem_base + ((uint32_t)(quad * 32) << 16) + acc * PAIR_BN;
+      epilogue_row<PAIR_BN, EPI>(p, c.b, row, c.nt * PAIR_BN, t_addr);
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(mapa_shared(smem_u32(&tmem_empty[acc]), 0));
+      if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+    }
+  }
+
+  // Neither CTA leaves (or frees TMEM) while the other may still read its shared memory, write
+  // its TMEM or arrive on its barriers.
+  tc_fence_before();
+  __syncthreads();
+  cluster_arrive();
+  cluster_wait();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc_pair(tmem_base, PAIR_TMEM_COLS);
   }
   if (threadIdx.x == 0 && *abort_flag && p.status) atomicExch(p.status, STATUS_TIMEOUT_MBARRIER);
 }
@@ -365,19 +550,7 @@ static int sm_count() {
   return g_sm_count;
 }
 
-template <int BN, int EPI>
-static int launch_gemm_t(const GemmLaunch& g, cudaStream_t stream) {
-  using Cfg = GemmCfg<BN>;
-  static bool attr_set = false;
-  auto kern = gemm_bf16_kernel<BN, EPI>;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES);
-    if (e != cudaSuccess) {
-      set_last_cuda_error((int)e);
-      return XEMA_ECUDA;
-    }
-    attr_set = true;
-  }
+static GemmParams make_params(const GemmLaunch& g) {
   GemmParams p;
   p.bias = (const __nv_bfloat16*)g.bias;
   p.out = g.out;
@@ -399,11 +572,83 @@ static int launch_gemm_t(const GemmLaunch& g, cudaStream_t stream) {
   p.head_dim = g.head_dim;
   p.norm_cols = g.norm_cols;
   p.rms_eps = g.rms_eps;
+  return p;
+}
+
+template <int BN, int EPI>
+static int launch_gemm_t(const GemmLaunch& g, cudaStream_t stream) {
+  using Cfg = GemmCfg<BN>;
+  static bool attr_set = false;
+  auto kern = gemm_bf16_kernel<BN, EPI>;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES);
+    if (e != cudaSuccess) {
+      set_last_cuda_error((int)e);
+      return XEMA_ECUDA;
+    }
+    attr_set = true;
+  }
+  const GemmParams p = make_params(g);
   const int m_tiles = (g.rows + BM - 1) / BM;
   const long long tiles = (long long)g.batch * m_tiles * (g.N / BN);
   const int grid = (int)std::min<long long>(tiles, sm_count());
   kern<<<grid, GEMM_THREADS, Cfg::SMEM_BYTES, stream>>>(g.map_a, g.map_w, p);
   return check_launch();
+}
+
+template <int EPI>
+static int launch_gemm_pair_t(const GemmLaunch& g, cudaStream_t stream) {
+  static bool attr_set = false;
+  auto kern = gemm_bf16_pair_kernel<EPI>;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, PAIR_SMEM_BYTES);
+    if (e != cudaSuccess) {
+      set_last_cuda_error((int)e);
+      return XEMA_ECUDA;
+    }
+    attr_set = true;
+  }
+  // A persistent grid must be resident all at once: ask how many CTA pairs fit on the device
+  // (SMs are handed out to clusters in hardware groups, so it can be fewer than SMs / 2).
+  static int max_pairs = 0;
+  if (max_pairs == 0) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * (sm_count() / 2), 1, 1);
+    cfg.blockDim = dim3(GEMM_THREADS, 1, 1);
+    cfg.dynamicSmemBytes = PAIR_SMEM_BYTES;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = 2;
+    at[0].val.clusterDim.y = 1;
+    at[0].val.clusterDim.z = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    int n = 0;
+    cudaError_t e = cudaOccupancyMaxActiveClusters(&n, kern, &cfg);
+    if (e != cudaSuccess || n <= 0) {
+      set_last_cuda_error((int)e);
+      return XEMA_ECUDA;
+    }
+    max_pairs = std::min(n, sm_count() / 2);
+    if (getenv("XEMA_DEBUG")) fprintf(stderr, "[xema] resident CTA pairs: %d\n", n);
+  }
+  const GemmParams p = make_params(g);
+  const int m_tiles = (g.rows + 2 * BM - 1) / (2 * BM);
+  const long long tiles = (long long)g.batch * m_tiles * (g.N / PAIR_BN);
+  const int pairs = (int)std::min<long long>(tiles, max_pairs);
+  kern<<<2 * pairs, GEMM_THREADS, PAIR_SMEM_BYTES, stream>>>(g.map_a, g.map_w, p);
+  return check_launch();
+}
+
+static int launch_gemm_pair(const GemmLaunch& g, cudaStream_t stream) {
+  switch (g.epilogue) {
+    case XEMA_EPI_BIAS: return launch_gemm_pair_t<XEMA_EPI_BIAS>(g, stream);
+    case XEMA_EPI_BIAS_GELU: return launch_gemm_pair_t<XEMA_EPI_BIAS_GELU>(g, stream);
+    case XEMA_EPI_GATE_RES_F32: return launch_gemm_pair_t<XEMA_EPI_GATE_RES_F32>(g, stream);
+    case XEMA_EPI_GATE_RES_BF16: return launch_gemm_pair_t<XEMA_EPI_GATE_RES_BF16>(g, stream);
+    case XEMA_EPI_BIAS_NORM_ROPE: return launch_gemm_pair_t<XEMA_EPI_BIAS_NORM_ROPE>(g, stream);
+    default: return XEMA_EINVAL;
+  }
 }
 
 template <int BN>
@@ -420,7 +665,7 @@ static int launch_gemm_bn(const GemmLaunch& g, cudaStream_t stream) {
 
 int launch_gemm(const GemmLaunch& g, cudaStream_t stream) {
   if (g.rows == 0 || g.batch == 0) return XEMA_OK;
-  if (g.block_n == 256) return launch_gemm_bn<256>(g, stream);
+  if (g.block_n == 256) return launch_gemm_pair(g, stream);
   if (g.block_n == 128) return launch_gemm_bn<128>(g, stream);
   return XEMA_EINVAL;
 }
@@ -445,7 +690,8 @@ int gemm_prepare(GemmLaunch* g, const void* a, long long lda, long long a_batch_
   g->block_n = (g->N % 256 == 0) ? 256 : 128;
   int rc = encode_tmap_bf16(&g->map_a, a, g->K, g->rows > 0 ? g->rows : 1, g->batch, lda, a_batch_rows, BM);
   if (rc) return rc;
-  return encode_tmap_bf16(&g->map_w, w, g->K, g->N, 1, ldw, g->N, g->block_n);
+  // the pair kernel (N % 256 == 0) loads the W tile as two 128-row halves, one per CTA
+  return encode_tmap_bf16(&g->map_w, w, g->K, g->N, 1, ldw, g->N, 128);
 }
 
 }  // namespace xema
