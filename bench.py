@@ -86,16 +86,40 @@ def attention_traffic_bytes(t, rows: int) -> float:
 
 
 class ClockSampler:
-    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    """Samples SM clock, power and throttle reasons of one GPU while the timed region runs: NVML
+    polled every few milliseconds from a thread (read-only queries), else nvidia-smi at its
+    fastest period."""
 
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
+    NVML_REASONS = ((0x8, "hw_slowdown"), (0x40, "hw_thermal_slowdown"), (0x20, "sw_thermal_slowdown"),
+                    (0x4, "sw_power_cap"))
 
     def __init__(self, index: int):
-        self.index, self.rows, self.proc = index, [], None
+        self.index, self.rows, self.proc, self.nvml, self.stop_flag = index, [], None, None, False
+        self.samples = []
+
+    def _nvml_handle(self):
+        import pynvml
+        pynvml.nvmlInit()
+        try:
+            import torch
+            uuid = str(torch.cuda.get_device_properties(self.index).uuid)
+            h = pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + uuid) if not uuid.startswith("GPU-") else uuid)
+        except Exception:
+            h = pynvml.nvmlDeviceGetHandleByIndex(self.index)
+        return pynvml, h
 
     def start(self):
+        try:
+            self.nvml, self.handle = self._nvml_handle()
+            self.sm_max = float(self.nvml.nvmlDeviceGetMaxClockInfo(self.handle, self.nvml.NVML_CLOCK_SM))
+            self.thread = threading.Thread(target=self._poll, daemon=True)
+            self.thread.start()
+            return
+        except Exception:
+            self.nvml = None
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
                                           "--format=csv,noheader,nounits", "-lms", "100"],
@@ -105,13 +129,32 @@ class ClockSampler:
         except Exception:
             self.proc = None
 
+    def _poll(self):
+        n, h = self.nvml, self.handle
+        while not self.stop_flag:
+            try:
+                self.samples.append((float(n.nvmlDeviceGetClockInfo(h, n.NVML_CLOCK_SM)),
+                                     n.nvmlDeviceGetPowerUsage(h) / 1000.0,
+                                     int(n.nvmlDeviceGetCurrentClocksEventReasons(h))))
+            except Exception:
+                pass
+            time.sleep(0.005)
+
     def _read(self):
         for line in self.proc.stdout:
             self.rows.append([c.strip() for c in line.split(",")])
 
     def stop(self) -> dict:
+        if self.nvml is not None:
+            self.stop_flag = True
+            self.thread.join(timeout=2)
+            sm = [s[0] for s in self.samples]
+            reasons = sorted({name for s in self.samples for bit, name in self.NVML_REASONS if s[2] & bit})
+            return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_min_mhz": min(sm) if sm else None,
+                    "sm_max_mhz": self.sm_max, "power_w_max": max((s[1] for s in self.samples), default=None),
+                    "samples": len(sm), "source": "nvml, 5 ms period", "reasons": reasons}
         if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no clock source available"]}
         time.sleep(0.15)
         self.proc.terminate()
         try:
@@ -131,7 +174,8 @@ class ClockSampler:
                 if v.lower().startswith("active"):
                     reasons.add(n)
         return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+                "power_w_max": max(power) if power else None, "samples": len(sm), "source": "nvidia-smi",
+                "reasons": sorted(reasons)}
 
 
 def oracle_inputs(t):
@@ -289,6 +333,17 @@ def main():
         e2e_step()
     e1.record(stream)
     barrier()
+    e2e_serial_ms = max_over_ranks(e0.elapsed_time(e1), dist, dev) / args.steps
+    # the same K steps with the copies of neighbouring steps overlapped with compute
+    done = sess.run_pipelined([x_host] * 3, [temb_host] * 3, [out_host] * 3, stream)
+    barrier()
+    done.synchronize()
+    e0.record(stream)
+    done = sess.run_pipelined([x_host] * args.steps, [temb_host] * args.steps, [out_host] * args.steps, stream)
+    stream.wait_event(done)
+    e1.record(stream)
+    barrier()
+    sess.check_status()
     e2e_ms = max_over_ranks(e0.elapsed_time(e1), dist, dev) / args.steps
     h2d = int(x_host.numel() * 2 + temb_host.numel() * 2)
     d2h = int(out_host.numel() * 2)
@@ -368,7 +423,11 @@ def main():
                    "parallelism": "replicas x%d" % world},
         "clocks": clocks,
         "e2e": {"value": whole_job_tflops(flops, world, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms,
-                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "how": "pinned host -> device -> pinned host every step; the copies of neighbouring steps "
+                       "overlap compute (BlockSession.run_pipelined)",
+                "staging_bytes_outside_arena": sess.staging_bytes,
+                "serial": {"value": whole_job_tflops(flops, world, e2e_serial_ms), "ms_per_step": e2e_serial_ms}},
         "gpu_launches": n_kernels * args.steps,
         "roofline": roofline,
         "tensor_ops": {"tflops": tensor_fl / (tensor_ms * 1e-3) / 1e12, "ms": tensor_ms,

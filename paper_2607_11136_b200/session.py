@@ -114,3 +114,60 @@ class BlockSession:
         code = int(self.status.item())
         if code != 0:
             raise xb.XemaError(xb.XEMA_ETIMEOUT, "device status word 0x%08x" % (code & 0xFFFFFFFF))
+
+    # ---- host-to-host pipeline ----------------------------------------------------------
+    def run_pipelined(self, x_hosts, temb_hosts, out_hosts, stream: Optional[torch.cuda.Stream] = None):
+        """One forward per (x, temb) pair of pinned host tensors, results into the pinned
+        `out_hosts`; the host->device copy of step i+1 and the device->host copy of step i-1
+        run on their own streams while step i computes.  The arena itself cannot take the next
+        input early (its input slot is reused inside the block), so the copies go through one
+        staging buffer per direction, outside the arena; `staging_bytes` says how large they
+        are.  Returns after everything was enqueued; synchronise `stream` and the returned
+        event before reading `out_hosts`."""
+        compute = stream or torch.cuda.current_stream(self.device)
+        if not hasattr(self, "_pipe"):
+            self._pipe = {
+                "h2d": torch.cuda.Stream(self.device), "d2h": torch.cuda.Stream(self.device),
+                "x": torch.empty_like(self.hid_in()), "temb": torch.empty_like(self.temb()),
+                "y": torch.empty_like(self.hid_out()),
+            }
+        pp = self._pipe
+        # staging input consumed by the arena copy / staging output read back by the host copy;
+        # carried over from an earlier call, whose last copies may still be in flight
+        in_free, out_free = pp.get("in_free"), pp.get("out_free")
+        if in_free is None:
+            in_free, out_free = torch.cuda.Event(), torch.cuda.Event()
+            in_free.record(compute)
+            out_free.record(compute)
+        done = None
+        for x_h, t_h, y_h in zip(x_hosts, temb_hosts, out_hosts):
+            ready = torch.cuda.Event()
+            with torch.cuda.stream(pp["h2d"]):
+                pp["h2d"].wait_event(in_free)
+                pp["x"].copy_(x_h.view(pp["x"].shape), non_blocking=True)
+                pp["temb"].copy_(t_h.view(pp["temb"].shape), non_blocking=True)
+                ready.record(pp["h2d"])
+            with torch.cuda.stream(compute):
+                compute.wait_event(ready)
+                self.hid_in().copy_(pp["x"], non_blocking=True)
+                self.temb().copy_(pp["temb"], non_blocking=True)
+                in_free = torch.cuda.Event()
+                in_free.record(compute)
+                self.forward(compute)
+                compute.wait_event(out_free)
+                pp["y"].copy_(self.hid_out(), non_blocking=True)
+                produced = torch.cuda.Event()
+                produced.record(compute)
+            with torch.cuda.stream(pp["d2h"]):
+                pp["d2h"].wait_event(produced)
+                y_h.view(pp["y"].shape).copy_(pp["y"], non_blocking=True)
+                out_free = torch.cuda.Event()
+                out_free.record(pp["d2h"])
+                done = out_free
+        pp["in_free"], pp["out_free"] = in_free, out_free
+        return done
+
+    @property
+    def staging_bytes(self) -> int:
+        t = self.template
+        return 2 * (2 * t.batch * self.seq * t.hidden) + 2 * t.batch * t.temb_dim

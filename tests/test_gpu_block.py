@@ -277,3 +277,31 @@ def test_bounded_wait_gives_up_and_reports():
     s.forward()
     ref = ob.block_forward(t, _f64(w), bits_to_f64(x), bits_to_f64(temb))["y"]
     assert_close(bits_to_f64(s.output_bits()), ref, "block after a timed-out wait")
+
+
+def test_pipelined_host_to_host_equals_serial(tiny_case):
+    """run_pipelined (copies of neighbouring steps overlapped with compute) returns, for every
+    step, the bits of a plain set_inputs / forward / output_bits round trip."""
+    t, w, x, temb, ref = tiny_case
+    s = BlockSession(t, [w], chunks=(1, 1, 2))
+    rng = np.random.default_rng(5)
+    xs = [x] + [(x.astype(np.uint32) ^ (rng.integers(0, 2, x.shape, dtype=np.uint32) << 15)).astype(np.uint16)
+                for _ in range(4)]               # sign flips: still finite bf16 values
+    want = []
+    for xi in xs:
+        s.set_inputs(xi, temb)
+        s.forward()
+        want.append(s.output_bits().copy())
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).pin_memory()
+    x_h = [pin(xi) for xi in xs]
+    t_h = [pin(temb) for _ in xs]
+    y_h = [torch.empty_like(x_h[0]).pin_memory() for _ in xs]
+    for _ in range(2):                           # a second call reuses the staging buffers
+        done = s.run_pipelined(x_h, t_h, y_h)
+        done.synchronize()
+        torch.cuda.synchronize()
+        s.check_status()
+        for got, exp in zip(y_h, want):
+            assert np.array_equal(got.numpy().view(np.uint16).reshape(exp.shape), exp)
+    assert np.array_equal(want[0], _run(t, [w], x, temb, 1)[1])
+    assert s.staging_bytes == 2 * x.size * 2 + temb.size * 2
