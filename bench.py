@@ -75,14 +75,14 @@ def whole_job_tflops(flops_per_replica: float, world: int, ms: float) -> float:
 
 
 # DRAM traffic of one attention launch, from the ncu capture summarised in
-# profiles/attention_dh64_rows2222_keys17776_h48.md (2222 query rows): 256.7 MB read + written, of
+# profiles/attention_dh64_rows2222_keys17776_h48.md (2222 query rows): 254.4 MB read + written, of
 # which k and v (4*S*D bytes, independent of the number of query rows) are read once and the
 # rest scales with the query rows.
 def attention_traffic_bytes(t, rows: int) -> float:
     if (t.seq, t.hidden, t.head_dim) != (17776, 3072, 64):
         return None
     kv = 4.0 * t.seq * t.hidden
-    return kv + (256.7e6 - kv) * rows / 2222.0
+    return kv + (254.4e6 - kv) * rows / 2222.0
 
 
 class ClockSampler:

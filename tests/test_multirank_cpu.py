@@ -49,4 +49,4 @@ def test_single_process_needs_no_group():
     from xema_inputs import template
     t = template("cogvideox")
     assert abs(bench.block_flops(t) - 7.910e12) / 7.910e12 < 1e-3
-    assert bench.attention_traffic_bytes(t, 2222) == 256.7e6
+    assert bench.attention_traffic_bytes(t, 2222) == 254.4e6
