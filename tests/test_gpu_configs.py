@@ -120,3 +120,14 @@ def test_cogvideox_step_42_blocks_teacher_forced():
     s.set_inputs(x, temb)
     s.forward()
     assert np.array_equal(s.output_bits(), y_blocks)
+
+
+def test_allocator_replay_static_arena_never_exceeds_the_caching_allocator():
+    """The trace replayed as torch.empty / del through PyTorch's caching allocator reserves at
+    least the active peak; the planned arena equals the active peak on this template."""
+    from paper_2607_11136_b200.alloc_replay import replay
+    r = replay([("cogvideox", (1, 1, 2)), ("flux", 1), ("cogvideox", 8)], rounds=2)
+    assert r["static_arena_bytes"] == r["active_peak_bytes"] == 600760320
+    assert r["active_peak_bytes"] <= r["torch_allocated_peak_bytes"] <= r["torch_reserved_peak_bytes"]
+    assert r["utilisation_static"] == 1.0 and 0.5 < r["utilisation_torch"] <= 1.0
+    torch.cuda.empty_cache()

@@ -159,3 +159,27 @@ def test_phase_chunks_for_budget_bit_exact():
             assert got == o_arena.phase_chunks_for_budget(t, budget, 16), (name, budget)
     with pytest.raises(xb.XemaError):
         xb.xema_phase_chunks_for_budget(xb.make_config(template("tiny")), 1 << 30, 0)
+
+
+def test_alloc_replay_event_order_reproduces_the_live_trace():
+    """The allocator replay issues frees before allocations at an op and its running byte count
+    equals the oracle's live-byte trace at every op."""
+    from paper_2607_11136_b200.alloc_replay import alloc_events, parse_item
+    assert parse_item("cogvideox:1,1,2") == ("cogvideox", (1, 1, 2)) and parse_item("flux:3") == ("flux", 3)
+    assert parse_item("tiny") == ("tiny", 1)
+    t = template("tiny")
+    for counts in [(1, 1, 1), (2, 1, 3), (3, 3, 3)]:
+        tensors, n_ops = o_trace.trace(t, counts)
+        live = o_arena.live_per_op(tensors, n_ops)
+        ev = alloc_events(tensors, n_ops)
+        assert sorted(i for _, k, i in ev if k == "alloc") == list(range(len(tensors)))
+        assert sorted(i for _, k, i in ev if k == "free") == list(range(len(tensors)))
+        cur, seen = 0, {}
+        for op, kind, i in ev:
+            cur += tensors[i]["bytes"] if kind == "alloc" else -tensors[i]["bytes"]
+            seen[op] = cur                      # value after the last event of this op
+        got, last = [], 0
+        for op in range(n_ops):                 # ops without an event keep the running value
+            last = seen.get(op, last)
+            got.append(last)
+        assert got == live and cur == 0
