@@ -24,7 +24,8 @@
  *
  * Conventions
  *   - All functions return 0 (XEMA_OK) or a negative xema_status; nothing throws, aborts,
- *     allocates device memory, frees device memory or synchronises a stream or device.
+ *     allocates device memory, frees device memory or synchronises a stream or device
+ *     (one stated exception: the allocator plug-in's malloc / free entry points).
  *   - "host" / "device" is stated for every pointer.  Device pointers must belong to the
  *     CUDA device that is current when the function is called.
  *   - Linear layers are y = x W^T + b with W stored [out, in] row-major, bf16.
@@ -313,6 +314,47 @@ int xema_op_attention(const void* q, int64_t ldq, int64_t q_batch_rows, const vo
                       int64_t ldkv, int64_t kv_batch_rows, void* o, float* lse, int32_t batch,
                       int32_t rows, int32_t keys, int32_t heads, int32_t head_dim, void* status_dev,
                       void* stream);
+
+/* ---- allocator plug-in ------------------------------------------------------------------ */
+/* The paper's run-time mechanism for code that is not this library's own kernels (section
+ * "Static memory runtime"; implementation: PyTorch's CUDAPluggableAllocator): a framework hands
+ * every device allocation and release to xema_pluggable_malloc / xema_pluggable_free; one
+ * step is recorded, its requests are laid out by xema_plan_arena, and from then on the k-th
+ * request of a step is answered by a table lookup, arena + offset[k].
+ *
+ * These are the only entry points of the library that call cudaMalloc / cudaFree (in the
+ * pass-through and record modes, and for requests that do not match the plan); they never
+ * synchronise.  All state is process-wide and guarded by one mutex.
+ *
+ * Lifetimes are measured on a clock that ticks once per allocation: request i is born at its
+ * own tick and dies at the tick of the first allocation after its release (at the end of the
+ * recording if it was never released).  Everything a recorded step allocates must be released
+ * before the next replayed step starts, because the next step gets the same addresses. */
+enum { XEMA_ALLOC_PASSTHROUGH = 0, XEMA_ALLOC_RECORD = 1, XEMA_ALLOC_REPLAY = 2 };
+
+/* Signatures CUDAPluggableAllocator expects.  size in bytes; device and stream are ignored
+ * (the current device is used).  malloc returns NULL on failure (see xema_last_cuda_error)
+ * and for size 0 (empty requests are not part of a recording); free of an address inside the
+ * planned arena does nothing. */
+void* xema_pluggable_malloc(ptrdiff_t size, int device, void* stream);
+void xema_pluggable_free(void* ptr, ptrdiff_t size, int device, void* stream);
+
+/* Switches mode.  -> RECORD clears the previous recording and plan; leaving RECORD closes the
+ * lifetimes of requests still live; -> REPLAY needs a plan (XEMA_ESTATE otherwise) and starts
+ * at request 0. */
+int xema_pluggable_mode(int mode);
+/* The recording as tensors (bytes rounded up to 256, birth, death; name "req<i>") in request
+ * order, for xema_plan_arena.  out: host, capacity cap; *n_requests and *n_events (host) are
+ * always written; XEMA_ENOSPC when cap is too small; XEMA_ESTATE while still recording. */
+int xema_pluggable_recorded(xema_tensor* out, size_t cap, size_t* n_requests, uint32_t* n_events);
+/* Installs the plan: arena_dev (device, 256-aligned, caller-owned, must outlive replay),
+ * offsets (host, one per recorded request, multiples of 256).  Only in pass-through mode. */
+int xema_pluggable_set_plan(void* arena_dev, uint64_t arena_bytes, const uint64_t* offsets, size_t n);
+/* Replay mode: the next request is request 0 again. */
+int xema_pluggable_step_begin(void);
+/* Counters since load: requests served from the arena, requests that fell back to cudaMalloc
+ * in replay mode, and the index the next request will be matched against.  Any may be NULL. */
+int xema_pluggable_stats(uint64_t* served, uint64_t* fallback, uint64_t* next_index);
 
 /* ---- diagnostics ------------------------------------------------------------------------ */
 /* Every wait inside the kernels (on an mbarrier fed by TMA, by the tensor pipe or by another

@@ -28,7 +28,10 @@ EXPORTS = (
     "xema_plan_launch_count", "xema_forward_prefix", "xema_forward_range", "xema_plan_op", "xema_op_mod", "xema_op_ln_modulate",
     "xema_op_rmsnorm_rope", "xema_op_gemm", "xema_op_attention", "xema_strerror",
     "xema_last_cuda_error", "xema_version", "xema_selftest_wait_timeout",
+    "xema_pluggable_malloc", "xema_pluggable_free", "xema_pluggable_mode", "xema_pluggable_recorded",
+    "xema_pluggable_set_plan", "xema_pluggable_step_begin", "xema_pluggable_stats",
 )
+ALLOC_PASSTHROUGH, ALLOC_RECORD, ALLOC_REPLAY = 0, 1, 2
 
 
 class XemaError(RuntimeError):
@@ -90,6 +93,11 @@ def lib() -> C.CDLL:
             "xema_plan_create_phases": [P(xema_config), P(i32), P(vp)],
             "xema_plan_phase_chunks": [vp, P(i32)],
             "xema_plan_arena": [P(xema_tensor), sz, P(u64), P(u64), P(u64)],
+            "xema_pluggable_mode": [C.c_int],
+            "xema_pluggable_recorded": [P(xema_tensor), sz, P(sz), P(u32)],
+            "xema_pluggable_set_plan": [vp, u64, P(u64), sz],
+            "xema_pluggable_step_begin": [],
+            "xema_pluggable_stats": [P(u64), P(u64), P(u64)],
             "xema_chunks_for_budget": [P(xema_config), u64, i32, P(i32), P(u64)],
             "xema_rope_table": [P(xema_config), vp],
             "xema_plan_create": [P(xema_config), i32, P(vp)],
@@ -214,6 +222,39 @@ def xema_chunks_for_budget(cfg: xema_config, budget_bytes: int, max_chunks: int)
         return None, peak.value
     _check(rc, "xema_chunks_for_budget")
     return ch.value, peak.value
+
+
+def xema_pluggable_mode(mode: int):
+    _check(lib().xema_pluggable_mode(mode), "xema_pluggable_mode")
+
+
+def xema_pluggable_recorded():
+    """-> (list of tensor dicts in request order, n_events)"""
+    n, ev = C.c_size_t(0), C.c_uint32(0)
+    rc = lib().xema_pluggable_recorded(None, 0, C.byref(n), C.byref(ev))
+    if rc != XEMA_ENOSPC:
+        _check(rc, "xema_pluggable_recorded")
+    if n.value == 0:
+        return [], ev.value
+    arr = (xema_tensor * n.value)()
+    _check(lib().xema_pluggable_recorded(arr, n.value, C.byref(n), C.byref(ev)), "xema_pluggable_recorded")
+    return [_tensor_dict(t) for t in arr], ev.value
+
+
+def xema_pluggable_set_plan(arena_ptr: int, arena_bytes: int, offsets: Sequence[int]):
+    offs = (C.c_uint64 * max(len(offsets), 1))(*offsets)
+    _check(lib().xema_pluggable_set_plan(arena_ptr, arena_bytes, offs, len(offsets)), "xema_pluggable_set_plan")
+
+
+def xema_pluggable_step_begin():
+    _check(lib().xema_pluggable_step_begin(), "xema_pluggable_step_begin")
+
+
+def xema_pluggable_stats():
+    """-> (served from the arena, fell back to cudaMalloc, index of the next request)"""
+    a, b, c = C.c_uint64(0), C.c_uint64(0), C.c_uint64(0)
+    _check(lib().xema_pluggable_stats(C.byref(a), C.byref(b), C.byref(c)), "xema_pluggable_stats")
+    return a.value, b.value, c.value
 
 
 def xema_rope_table(cfg: xema_config) -> np.ndarray:

@@ -12,7 +12,7 @@ CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "build")
 LIB = os.path.join(HERE, "libxema.so")
 
-SOURCES = ["planner.cpp", "elementwise.cu", "gemm.cu", "attention.cu", "attention_dh64.cu", "runtime.cu", "static_arena.cu", "selftest.cu"]
+SOURCES = ["planner.cpp", "elementwise.cu", "gemm.cu", "attention.cu", "attention_dh64.cu", "runtime.cu", "static_arena.cu", "selftest.cu", "pluggable.cpp"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-Wall", "--expt-relaxed-constexpr"]
 
