@@ -306,6 +306,7 @@ def main():
     sess.check_status()
     total_ms = max_over_ranks(ev[0][0].elapsed_time(ev[-1][n_launch]), dist, dev)
     ms_per_step = total_ms / args.steps
+    step_ms = sorted(ev[k][0].elapsed_time(ev[k][n_launch]) for k in range(args.steps))
     value = whole_job_tflops(flops, world, ms_per_step)
 
     per_op = {}
@@ -410,7 +411,8 @@ def main():
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "ms_median": step_ms[len(step_ms) // 2],
+        "ms_min": step_ms[0], "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": args.workload, "batch": t.batch, "tokens": t.seq, "hidden": t.hidden,
                    "heads": t.heads, "head_dim": t.head_dim, "ffn": t.ffn, "n_blocks": t.n_blocks,
