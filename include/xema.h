@@ -155,6 +155,30 @@ int xema_trace_phases(const xema_config* cfg, const int32_t chunks[3], xema_tens
 int xema_phase_chunks_for_budget(const xema_config* cfg, uint64_t budget_bytes,
                                  int32_t max_chunks, int32_t chunks[3], uint64_t* peak_bytes);
 
+/* Temporary serialization (section "Applying Mitigation Only Where Needed", paragraph
+ * "Temporary serialization"; "Memory mitigation primitives": only the planned steps are split
+ * into sub-batches, which rejoin afterwards).  A phase can be split along the batch instead of
+ * along the rows: piece c of C then covers batch elements [floor(c*B/C), floor((c+1)*B/C)) and
+ * all S rows (1 <= C <= B); the full-size tensors kv, res and hid are where the sub-batches
+ * rejoin.  chunks[p] pieces along axis[p] for phase p. */
+enum { XEMA_SPLIT_ROWS = 0, XEMA_SPLIT_BATCH = 1 };
+typedef struct xema_mitigation {
+  int32_t chunks[3]; /* pieces of the key/value, attention and feed-forward phase            */
+  int32_t axis[3];   /* XEMA_SPLIT_ROWS or XEMA_SPLIT_BATCH per phase                         */
+} xema_mitigation;
+
+/* xema_trace_phases with a split axis per phase (all XEMA_SPLIT_ROWS gives the same trace).
+ * XEMA_EINVAL: a count outside [1, S] (rows) or [1, B] (batch), or an unknown axis. */
+int xema_trace_mitigated(const xema_config* cfg, const xema_mitigation* m, xema_tensor* out,
+                         size_t cap, size_t* n_tensors, uint32_t* n_ops);
+
+/* The search of xema_phase_chunks_for_budget where, at every step, a phase that is split
+ * C > 1 ways is split into sub-batches while C <= B and into row chunks beyond that.  *m
+ * (host) receives counts and axes (axis of an unsplit phase: XEMA_SPLIT_ROWS); on
+ * XEMA_EBUDGET the counts are zeroed and *peak_bytes is the smallest reserved peak seen. */
+int xema_mitigation_for_budget(const xema_config* cfg, uint64_t budget_bytes, int32_t max_chunks,
+                               xema_mitigation* m, uint64_t* peak_bytes);
+
 /* RoPE table for the template: host_out (host) receives S * (dh/2) * 2 floats laid out
  * [token][pair][cos, sin]; angle = position * rope_base^(-2j/d) inside each of the three
  * sections (t, h, w), evaluated in double precision and rounded once.  Text tokens sit at
@@ -177,6 +201,9 @@ int xema_plan_info(const xema_plan* plan, uint64_t* peak_bytes, uint64_t* max_li
                    size_t* n_tensors, uint32_t* n_ops, int32_t* chunks);
 /* The plan's per-phase chunk counts; chunks: host, 3 entries. */
 int xema_plan_phase_chunks(const xema_plan* plan, int32_t chunks[3]);
+/* Plan with a split axis per phase (see xema_trace_mitigated), and the plan's counts and axes. */
+int xema_plan_create_mitigated(const xema_config* cfg, const xema_mitigation* m, xema_plan** out);
+int xema_plan_mitigation(const xema_plan* plan, xema_mitigation* m);
 /* Offset and (256-rounded) size of a tensor by name, e.g. "hid0", "temb", "hid1", "res0". */
 int xema_plan_tensor(const xema_plan* plan, const char* name, uint64_t* offset, uint64_t* bytes);
 /* Copy of the plan's tensor i and its offset. */

@@ -138,6 +138,35 @@ def phase_chunks_for_budget(t, budget_bytes, max_chunks):
                 return None, smallest
 
 
+def serialization_axes(t, counts):
+    """Temporary serialization where the batch allows it: a phase split C > 1 ways is split into
+    sub-batches when C <= B, into row chunks otherwise (and when it is not split at all)."""
+    return tuple(_trace.SPLIT_BATCH if 1 < c <= t.batch else _trace.SPLIT_ROWS for c in counts)
+
+
+def mitigation_for_budget(t, budget_bytes, max_chunks):
+    """phase_chunks_for_budget with the split axis chosen by serialization_axes at every step.
+    Returns ((C_A, C_B, C_C), axes, reserved peak) or (None, None, smallest reserved peak seen)."""
+    counts = [1, 1, 1]
+    smallest = None
+    limit = min(max_chunks, t.seq)
+    while True:
+        axes = serialization_axes(t, counts)
+        tensors, n_ops = _trace.trace(t, tuple(counts), axes)
+        _, peak = plan_arena(tensors)
+        smallest = peak if smallest is None else min(smallest, peak)
+        live = live_per_op(tensors, n_ops)
+        over = {phase_of_op(t, counts, op) for op, b in enumerate(live) if b > budget_bytes}
+        if not over:
+            if peak <= budget_bytes:
+                return tuple(counts), axes, peak
+            over = {phase_of_op(t, counts, max(range(n_ops), key=lambda op: (live[op], -op)))}
+        for ph in sorted(over):
+            counts[ph] += 1
+            if counts[ph] > limit:
+                return None, None, smallest
+
+
 def chunks_for_budget(t, budget_bytes, max_chunks):
     """Returns (chunks, peak) for the first C in 1..max_chunks whose arena peak fits,
     or (None, smallest peak seen) when none does."""

@@ -170,15 +170,30 @@ def block_forward(t, W, x, temb, rows=None, row_block=2048, keep=False):
     return out
 
 
-def block_forward_chunked(t, W, x, temb, chunks):
+def block_forward_chunked(t, W, x, temb, chunks, axes=(0, 0, 0)):
     """The same block evaluated in the chunked three-phase order the library uses
     (all KV chunks; then Q/attention/projection per chunk; then the FFN per chunk),
     chunk c covering rows [floor(c S / C), floor((c+1) S / C)); `chunks` is one count or
-    a per-phase triple.  Used to show that chunking is lossless; not a second definition."""
+    a per-phase triple.  A phase whose axis is 1 is split into sub-batches instead (piece c =
+    batch elements [floor(c B / C), floor((c+1) B / C)), all rows).  Used to show that either
+    split is lossless; not a second definition."""
     x = np.asarray(x, F64)
     B, S, D = x.shape
     H, dh = t.heads, t.head_dim
     ca, cb, cc = (chunks, chunks, chunks) if isinstance(chunks, int) else chunks
+    if any(axes):
+        # a sub-batch piece holds whole batch elements: evaluate every element of the piece with
+        # that phase unchunked along the rows
+        y = np.empty((B, S, D))
+        lse = np.empty((B, H, S))
+        cuts = [[c * B // C for c in range(C + 1)] if ax else None for C, ax in zip((ca, cb, cc), axes)]
+        for b in range(B):
+            counts = tuple(1 if ax else C for C, ax in zip((ca, cb, cc), axes))
+            assert all(cut is None or any(cut[i] <= b < cut[i + 1] for i in range(len(cut) - 1)) for cut in cuts)
+            tb = t.with_(batch=1)
+            out = block_forward_chunked(tb, W, x[b:b + 1], np.asarray(temb)[b:b + 1], counts)
+            y[b], lse[b] = out["y"][0], out["lse"][0]
+        return {"y": y, "lse": lse}
     rows_of = lambda C: [c * S // C for c in range(C + 1)]
     shift1, scale1, gate1, shift2, scale2, gate2 = modulation(t, W, temb)
     ang = rope_angles(t)

@@ -13,6 +13,10 @@ Op order of one block with C sequence chunks (1 + 11 C ops):
     for c: LN1B_c, Q_c, QROPE_c, ATTN_c, PROJ_c
     for c: LN2_c, FFN1_c, FFN2_c
 Chunk c covers token rows [floor(c S / C), floor((c+1) S / C)).
+
+A phase may instead be split along the batch ("temporary serialization": only the planned steps
+are split into sub-batches, which rejoin in the full-size tensors afterwards): piece c of C then
+covers batch elements [floor(c B / C), floor((c+1) B / C)) and all S rows.
 """
 from __future__ import annotations
 
@@ -60,18 +64,34 @@ def phase_counts(chunks):
     return (ca, cb, cc)
 
 
-def trace(t, chunks):
+SPLIT_ROWS, SPLIT_BATCH = 0, 1
+
+
+def piece_elems(t, C, axis):
+    """Token-row count times batch count of every piece of a phase split C ways along `axis`."""
+    if axis == SPLIT_BATCH:
+        b = chunk_rows(t.batch, C)
+        return [(b[c + 1] - b[c]) * t.seq for c in range(C)]
+    r = chunk_rows(t.seq, C)
+    return [t.batch * (r[c + 1] - r[c]) for c in range(C)]
+
+
+def trace(t, chunks, axes=(SPLIT_ROWS, SPLIT_ROWS, SPLIT_ROWS)):
     """Returns (tensors, n_ops).  tensors: list of dicts with name, kind, dtype, block,
     chunk, bytes (rounded up to 256), birth, death -- in id order (first birth, then
     table row).  `chunks` is an int or a per-phase triple (see phase_counts); with a triple
     the op list is MOD; C_A x (LN1A, KV, KROPE); C_B x (LN1B, Q, QROPE, ATTN, PROJ);
-    C_C x (LN2, FFN1, FFN2) -- chunking applied only where the trace needs it."""
+    C_C x (LN2, FFN1, FFN2) -- chunking applied only where the trace needs it.  `axes` says per
+    phase whether its pieces are row chunks (all batch elements) or sub-batches (all rows)."""
     B, S, D, H, F, Dt = t.batch, t.seq, t.hidden, t.heads, t.ffn, t.temb_dim
     CA, CB, CC = phase_counts(chunks)
     L = t.n_blocks
-    if min(CA, CB, CC) < 1 or max(CA, CB, CC) > S:
-        raise ValueError("chunks must be in [1, S]")
-    rA, rB, rC = chunk_rows(S, CA), chunk_rows(S, CB), chunk_rows(S, CC)
+    for C, ax in zip((CA, CB, CC), axes):
+        if ax not in (SPLIT_ROWS, SPLIT_BATCH):
+            raise ValueError("axis must be 0 (rows) or 1 (batch)")
+        if C < 1 or C > (B if ax == SPLIT_BATCH else S):
+            raise ValueError("chunks must be in [1, S] (rows) or [1, B] (batch)")
+    eA, eB, eC = (piece_elems(t, C, ax) for C, ax in zip((CA, CB, CC), axes))
     rec = _Recorder()
 
     def meta(base, nbytes, kind, dtype, block, chunk=-1):
@@ -90,26 +110,26 @@ def trace(t, chunks):
         m_nxt = (nxt, meta("hid", u, KIND_OUTPUT if l + 1 == L else KIND_FULL, DTYPE_BF16, l + 1))
         rec.op(reads=["temb"], writes=[m_mod])                                   # MOD
         for c in range(CA):
-            n = rA[c + 1] - rA[c]
-            h1a = (f"h1a{l}_{c}", meta("h1a", 2 * B * n * D, KIND_CHUNK, DTYPE_BF16, l, c))
+            n = eA[c]
+            h1a = (f"h1a{l}_{c}", meta("h1a", 2 * n * D, KIND_CHUNK, DTYPE_BF16, l, c))
             rec.op(reads=[hid, mod], writes=[h1a])                               # LN1A
             rec.op(reads=[h1a[0]], writes=[m_kv])                                # KV
             rec.op(reads=[kv], writes=[m_kv])                                    # KROPE (in place)
         for c in range(CB):
-            n = rB[c + 1] - rB[c]
-            h1b = (f"h1b{l}_{c}", meta("h1b", 2 * B * n * D, KIND_CHUNK, DTYPE_BF16, l, c))
-            q = (f"q{l}_{c}", meta("q", 2 * B * n * D, KIND_CHUNK, DTYPE_BF16, l, c))
-            o = (f"o{l}_{c}", meta("o", 2 * B * n * D, KIND_CHUNK, DTYPE_BF16, l, c))
-            lse = (f"lse{l}_{c}", meta("lse", 4 * B * H * n, KIND_CHUNK, DTYPE_F32, l, c))
+            n = eB[c]
+            h1b = (f"h1b{l}_{c}", meta("h1b", 2 * n * D, KIND_CHUNK, DTYPE_BF16, l, c))
+            q = (f"q{l}_{c}", meta("q", 2 * n * D, KIND_CHUNK, DTYPE_BF16, l, c))
+            o = (f"o{l}_{c}", meta("o", 2 * n * D, KIND_CHUNK, DTYPE_BF16, l, c))
+            lse = (f"lse{l}_{c}", meta("lse", 4 * H * n, KIND_CHUNK, DTYPE_F32, l, c))
             rec.op(reads=[hid, mod], writes=[h1b])                               # LN1B
             rec.op(reads=[h1b[0]], writes=[q])                                   # Q
             rec.op(reads=[q[0]], writes=[q])                                     # QROPE (in place)
             rec.op(reads=[q[0], kv], writes=[o, lse])                            # ATTN
             rec.op(reads=[o[0], hid, mod], writes=[m_res])                       # PROJ
         for c in range(CC):
-            n = rC[c + 1] - rC[c]
-            h2 = (f"h2{l}_{c}", meta("h2", 2 * B * n * D, KIND_CHUNK, DTYPE_BF16, l, c))
-            g = (f"g{l}_{c}", meta("g", 2 * B * n * F, KIND_CHUNK, DTYPE_BF16, l, c))
+            n = eC[c]
+            h2 = (f"h2{l}_{c}", meta("h2", 2 * n * D, KIND_CHUNK, DTYPE_BF16, l, c))
+            g = (f"g{l}_{c}", meta("g", 2 * n * F, KIND_CHUNK, DTYPE_BF16, l, c))
             rec.op(reads=[res, mod], writes=[h2])                                # LN2
             rec.op(reads=[h2[0]], writes=[g])                                    # FFN1
             rec.op(reads=[g[0], res, mod], writes=[m_nxt])                       # FFN2

@@ -20,9 +20,9 @@ EPI_BIAS, EPI_BIAS_GELU, EPI_GATE_RES_F32, EPI_GATE_RES_BF16, EPI_BIAS_NORM_ROPE
 
 EXPORTS = (
     "xema_trace", "xema_trace_phases", "xema_plan_arena", "xema_chunks_for_budget",
-    "xema_phase_chunks_for_budget", "xema_rope_table",
-    "xema_plan_create", "xema_plan_create_phases", "xema_plan_destroy", "xema_plan_info",
-    "xema_plan_phase_chunks", "xema_plan_tensor",
+    "xema_phase_chunks_for_budget", "xema_trace_mitigated", "xema_mitigation_for_budget", "xema_rope_table",
+    "xema_plan_create", "xema_plan_create_phases", "xema_plan_create_mitigated", "xema_plan_destroy",
+    "xema_plan_info", "xema_plan_phase_chunks", "xema_plan_mitigation", "xema_plan_tensor",
     "xema_plan_tensor_at", "xema_plan_bind", "xema_block_forward", "xema_step_forward",
     "xema_block_forward_static",
     "xema_plan_launch_count", "xema_forward_prefix", "xema_forward_range", "xema_plan_op", "xema_op_mod", "xema_op_ln_modulate",
@@ -32,6 +32,11 @@ EXPORTS = (
     "xema_pluggable_set_plan", "xema_pluggable_step_begin", "xema_pluggable_stats",
 )
 ALLOC_PASSTHROUGH, ALLOC_RECORD, ALLOC_REPLAY = 0, 1, 2
+SPLIT_ROWS, SPLIT_BATCH = 0, 1
+
+
+class xema_mitigation(C.Structure):
+    _fields_ = [("chunks", C.c_int32 * 3), ("axis", C.c_int32 * 3)]
 
 
 class XemaError(RuntimeError):
@@ -91,6 +96,10 @@ def lib() -> C.CDLL:
             "xema_trace_phases": [P(xema_config), P(i32), P(xema_tensor), sz, P(sz), P(u32)],
             "xema_phase_chunks_for_budget": [P(xema_config), u64, i32, P(i32), P(u64)],
             "xema_plan_create_phases": [P(xema_config), P(i32), P(vp)],
+            "xema_trace_mitigated": [P(xema_config), P(xema_mitigation), P(xema_tensor), sz, P(sz), P(u32)],
+            "xema_mitigation_for_budget": [P(xema_config), u64, i32, P(xema_mitigation), P(u64)],
+            "xema_plan_create_mitigated": [P(xema_config), P(xema_mitigation), P(vp)],
+            "xema_plan_mitigation": [vp, P(xema_mitigation)],
             "xema_plan_phase_chunks": [vp, P(i32)],
             "xema_plan_arena": [P(xema_tensor), sz, P(u64), P(u64), P(u64)],
             "xema_pluggable_mode": [C.c_int],
@@ -202,6 +211,36 @@ def xema_phase_chunks_for_budget(cfg: xema_config, budget_bytes: int, max_chunks
     return tuple(c3), peak.value
 
 
+def _mitigation(chunks, axes):
+    m = xema_mitigation()
+    for i in range(3):
+        m.chunks[i], m.axis[i] = int(chunks[i]), int(axes[i])
+    return m
+
+
+def xema_trace_mitigated(cfg: xema_config, chunks, axes):
+    """chunks = (C_A, C_B, C_C), axes = per-phase SPLIT_ROWS / SPLIT_BATCH -> (tensor dicts, n_ops)"""
+    m = _mitigation(chunks, axes)
+    n, ops = C.c_size_t(0), C.c_uint32(0)
+    rc = lib().xema_trace_mitigated(C.byref(cfg), C.byref(m), None, 0, C.byref(n), C.byref(ops))
+    if rc != XEMA_ENOSPC:
+        _check(rc, "xema_trace_mitigated")
+    arr = (xema_tensor * n.value)()
+    _check(lib().xema_trace_mitigated(C.byref(cfg), C.byref(m), arr, n.value, C.byref(n), C.byref(ops)),
+           "xema_trace_mitigated")
+    return [_tensor_dict(t) for t in arr], ops.value
+
+
+def xema_mitigation_for_budget(cfg: xema_config, budget_bytes: int, max_chunks: int):
+    """-> ((C_A, C_B, C_C), axes, peak_bytes); counts and axes are None when nothing fits."""
+    m, peak = xema_mitigation(), C.c_uint64(0)
+    rc = lib().xema_mitigation_for_budget(C.byref(cfg), budget_bytes, max_chunks, C.byref(m), C.byref(peak))
+    if rc == XEMA_EBUDGET:
+        return None, None, peak.value
+    _check(rc, "xema_mitigation_for_budget")
+    return tuple(m.chunks), tuple(m.axis), peak.value
+
+
 def xema_plan_arena(tensors: Sequence[dict]):
     """tensors: dicts with bytes, birth, death -> (offsets, peak_bytes, max_live_bytes)"""
     n = len(tensors)
@@ -267,11 +306,16 @@ def xema_rope_table(cfg: xema_config) -> np.ndarray:
 class Plan:
     """Owner of an xema_plan handle."""
 
-    def __init__(self, cfg: xema_config, chunks):
-        """chunks: one count (xema_plan_create) or a per-phase triple (xema_plan_create_phases)."""
+    def __init__(self, cfg: xema_config, chunks, axes=None):
+        """chunks: one count (xema_plan_create) or a per-phase triple (xema_plan_create_phases);
+        with `axes` (per-phase SPLIT_ROWS / SPLIT_BATCH) xema_plan_create_mitigated."""
         self.cfg = cfg
         self._h = C.c_void_p()
-        if isinstance(chunks, int):
+        if axes is not None:
+            c3 = (chunks,) * 3 if isinstance(chunks, int) else chunks
+            _check(lib().xema_plan_create_mitigated(C.byref(cfg), C.byref(_mitigation(c3, axes)), C.byref(self._h)),
+                   "xema_plan_create_mitigated")
+        elif isinstance(chunks, int):
             _check(lib().xema_plan_create(C.byref(cfg), chunks, C.byref(self._h)), "xema_plan_create")
         else:
             _check(lib().xema_plan_create_phases(C.byref(cfg), _triple(chunks), C.byref(self._h)),
@@ -284,6 +328,9 @@ class Plan:
         c3 = (C.c_int32 * 3)()
         _check(lib().xema_plan_phase_chunks(self._h, c3), "xema_plan_phase_chunks")
         self.phase_chunks = tuple(c3)
+        m = xema_mitigation()
+        _check(lib().xema_plan_mitigation(self._h, C.byref(m)), "xema_plan_mitigation")
+        self.axes = tuple(m.axis)
         self._keep = None
 
     def close(self):

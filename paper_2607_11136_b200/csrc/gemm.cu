@@ -13,9 +13,6 @@
 //             other accumulator
 // A row's result depends only on (row, N, K): the K loop always runs in the same order and the
 // tile shape is chosen from N alone, so outputs are bit-identical however rows are chunked.
-#include <cstdio>
-#include <cstdlib>
-
 #include "kernels.h"
 #include "sm100.cuh"
 
@@ -630,7 +627,6 @@ static int launch_gemm_pair_t(const GemmLaunch& g, cudaStream_t stream) {
       return XEMA_ECUDA;
     }
     max_pairs = std::min(n, sm_count() / 2);
-    if (getenv("XEMA_DEBUG")) fprintf(stderr, "[xema] resident CTA pairs: %d\n", n);
   }
   const GemmParams p = make_params(g);
   const int m_tiles = (g.rows + 2 * BM - 1) / (2 * BM);

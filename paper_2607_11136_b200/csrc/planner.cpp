@@ -73,18 +73,31 @@ int build_trace(const xema_config& cfg, int32_t chunks, std::vector<xema_tensor>
 }
 
 int build_trace(const xema_config& cfg, const int32_t chunks[3], std::vector<xema_tensor>& out, uint32_t* n_ops) {
+  const int32_t axes[3] = {XEMA_SPLIT_ROWS, XEMA_SPLIT_ROWS, XEMA_SPLIT_ROWS};
+  return build_trace(cfg, chunks, axes, out, n_ops);
+}
+
+int build_trace(const xema_config& cfg, const int32_t chunks[3], const int32_t axes[3], std::vector<xema_tensor>& out,
+                uint32_t* n_ops) {
   int rc = validate_config(cfg);
   if (rc) return rc;
   const int64_t S = seq_len(cfg);
-  for (int i = 0; i < 3; ++i)
-    if (chunks[i] < 1 || chunks[i] > S) return XEMA_EINVAL;
+  for (int i = 0; i < 3; ++i) {
+    if (axes[i] != XEMA_SPLIT_ROWS && axes[i] != XEMA_SPLIT_BATCH) return XEMA_EINVAL;
+    if (chunks[i] < 1 || chunks[i] > (axes[i] == XEMA_SPLIT_BATCH ? (int64_t)cfg.batch : S)) return XEMA_EINVAL;
+  }
   const uint64_t B = cfg.batch, D = cfg.hidden, H = cfg.heads, F = cfg.ffn, Dt = cfg.temb_dim;
   const uint32_t CA = (uint32_t)chunks[0], CB = (uint32_t)chunks[1], CC = (uint32_t)chunks[2];
   const uint32_t L = (uint32_t)cfg.n_blocks;
   const uint32_t ops_per_block = 1 + 3 * CA + 5 * CB + 3 * CC;
   const uint32_t total_ops = L * ops_per_block;
   const uint64_t u = 2 * B * (uint64_t)S * D;
-  auto rows_of = [&](uint32_t c, uint32_t C) { return (uint64_t)((int64_t)(c + 1) * S / C - (int64_t)c * S / C); };
+  // rows x batch elements of piece c of a phase split C ways along its axis
+  auto elems_of = [&](uint32_t c, uint32_t C, int phase) {
+    if (axes[phase] == XEMA_SPLIT_BATCH)
+      return (uint64_t)((int64_t)(c + 1) * (int64_t)B / C - (int64_t)c * (int64_t)B / C) * (uint64_t)S;
+    return B * (uint64_t)((int64_t)(c + 1) * S / C - (int64_t)c * S / C);
+  };
 
   out.clear();
   out.reserve((size_t)L * (4 + 2 * CA + 4 * CB + 2 * CC) + 2);
@@ -101,24 +114,24 @@ int build_trace(const xema_config& cfg, const int32_t chunks[3], std::vector<xem
     }
     out.push_back(make("mod", l, -1, XEMA_KIND_FULL, XEMA_DTYPE_F32, 24 * B * D, op.mod(), op.ffn2(CC - 1) + 1));
     for (uint32_t c = 0; c < CA; ++c) {
-      uint64_t n = rows_of(c, CA);
-      out.push_back(make("h1a", l, c, XEMA_KIND_CHUNK, XEMA_DTYPE_BF16, 2 * B * n * D, op.ln1a(c), op.kv(c) + 1));
+      uint64_t n = elems_of(c, CA, 0);
+      out.push_back(make("h1a", l, c, XEMA_KIND_CHUNK, XEMA_DTYPE_BF16, 2 * n * D, op.ln1a(c), op.kv(c) + 1));
       if (c == 0)
         out.push_back(make("kv", l, -1, XEMA_KIND_FULL, XEMA_DTYPE_BF16, 2 * u, op.kv(0), op.attn(CB - 1) + 1));
     }
     for (uint32_t c = 0; c < CB; ++c) {
-      uint64_t n = rows_of(c, CB);
-      out.push_back(make("h1b", l, c, XEMA_KIND_CHUNK, XEMA_DTYPE_BF16, 2 * B * n * D, op.ln1b(c), op.q(c) + 1));
-      out.push_back(make("q", l, c, XEMA_KIND_CHUNK, XEMA_DTYPE_BF16, 2 * B * n * D, op.q(c), op.attn(c) + 1));
-      out.push_back(make("o", l, c, XEMA_KIND_CHUNK, XEMA_DTYPE_BF16, 2 * B * n * D, op.attn(c), op.proj(c) + 1));
-      out.push_back(make("lse", l, c, XEMA_KIND_CHUNK, XEMA_DTYPE_F32, 4 * B * H * n, op.attn(c), op.attn(c) + 1));
+      uint64_t n = elems_of(c, CB, 1);
+      out.push_back(make("h1b", l, c, XEMA_KIND_CHUNK, XEMA_DTYPE_BF16, 2 * n * D, op.ln1b(c), op.q(c) + 1));
+      out.push_back(make("q", l, c, XEMA_KIND_CHUNK, XEMA_DTYPE_BF16, 2 * n * D, op.q(c), op.attn(c) + 1));
+      out.push_back(make("o", l, c, XEMA_KIND_CHUNK, XEMA_DTYPE_BF16, 2 * n * D, op.attn(c), op.proj(c) + 1));
+      out.push_back(make("lse", l, c, XEMA_KIND_CHUNK, XEMA_DTYPE_F32, 4 * H * n, op.attn(c), op.attn(c) + 1));
       if (c == 0)
         out.push_back(make("res", l, -1, XEMA_KIND_FULL, XEMA_DTYPE_F32, 2 * u, op.proj(0), op.ffn2(CC - 1) + 1));
     }
     for (uint32_t c = 0; c < CC; ++c) {
-      uint64_t n = rows_of(c, CC);
-      out.push_back(make("h2", l, c, XEMA_KIND_CHUNK, XEMA_DTYPE_BF16, 2 * B * n * D, op.ln2(c), op.ffn1(c) + 1));
-      out.push_back(make("g", l, c, XEMA_KIND_CHUNK, XEMA_DTYPE_BF16, 2 * B * n * F, op.ffn1(c), op.ffn2(c) + 1));
+      uint64_t n = elems_of(c, CC, 2);
+      out.push_back(make("h2", l, c, XEMA_KIND_CHUNK, XEMA_DTYPE_BF16, 2 * n * D, op.ln2(c), op.ffn1(c) + 1));
+      out.push_back(make("g", l, c, XEMA_KIND_CHUNK, XEMA_DTYPE_BF16, 2 * n * F, op.ffn1(c), op.ffn2(c) + 1));
       if (c == 0) {
         // the next hidden state: written chunk by chunk from FFN2_0 on; read by the next
         // block up to its last PROJ, or kept to the end if it is the output
@@ -235,6 +248,14 @@ int chunks_for_budget(const xema_config& cfg, uint64_t budget, int32_t max_chunk
 // exceeds the budget afterwards, raise the phase that holds the op with the most live bytes.
 int phase_chunks_for_budget(const xema_config& cfg, uint64_t budget, int32_t max_chunks, int32_t chunks[3],
                             uint64_t* peak_out) {
+  int32_t axes[3];
+  return mitigation_for_budget(cfg, budget, max_chunks, false, chunks, axes, peak_out);
+}
+
+// The same search; with `serialize` a phase split C > 1 ways is split into sub-batches while
+// C <= B (temporary serialization) and into row chunks otherwise.
+int mitigation_for_budget(const xema_config& cfg, uint64_t budget, int32_t max_chunks, bool serialize,
+                          int32_t chunks[3], int32_t axes[3], uint64_t* peak_out) {
   int rc = validate_config(cfg);
   if (rc) return rc;
   if (max_chunks < 1) return XEMA_EINVAL;
@@ -245,7 +266,10 @@ int phase_chunks_for_budget(const xema_config& cfg, uint64_t budget, int32_t max
   std::vector<uint64_t> offs, live;
   while (true) {
     uint32_t n_ops = 0;
-    rc = build_trace(cfg, c, ts, &n_ops);
+    int32_t ax[3];
+    for (int i = 0; i < 3; ++i)
+      ax[i] = (serialize && c[i] > 1 && c[i] <= cfg.batch) ? XEMA_SPLIT_BATCH : XEMA_SPLIT_ROWS;
+    rc = build_trace(cfg, c, ax, ts, &n_ops);
     if (rc) return rc;
     offs.assign(ts.size(), 0);
     uint64_t peak = 0;
@@ -273,7 +297,10 @@ int phase_chunks_for_budget(const xema_config& cfg, uint64_t budget, int32_t max
     }
     if (!over[0] && !over[1] && !over[2]) {
       if (peak <= budget) {
-        for (int i = 0; i < 3; ++i) chunks[i] = c[i];
+        for (int i = 0; i < 3; ++i) {
+          chunks[i] = c[i];
+          axes[i] = ax[i];
+        }
         if (peak_out) *peak_out = peak;
         return XEMA_OK;
       }
@@ -283,6 +310,7 @@ int phase_chunks_for_budget(const xema_config& cfg, uint64_t budget, int32_t max
       if (!over[i]) continue;
       if (++c[i] > limit) {
         chunks[0] = chunks[1] = chunks[2] = 0;
+        axes[0] = axes[1] = axes[2] = XEMA_SPLIT_ROWS;
         if (peak_out) *peak_out = smallest;
         return XEMA_EBUDGET;
       }
@@ -360,6 +388,26 @@ int xema_phase_chunks_for_budget(const xema_config* cfg, uint64_t budget_bytes, 
                                  int32_t chunks[3], uint64_t* peak_bytes) {
   if (!cfg || !chunks) return XEMA_EINVAL;
   return xema::phase_chunks_for_budget(*cfg, budget_bytes, max_chunks, chunks, peak_bytes);
+}
+
+int xema_trace_mitigated(const xema_config* cfg, const xema_mitigation* m, xema_tensor* out, size_t cap,
+                         size_t* n_tensors, uint32_t* n_ops) {
+  if (!cfg || !m) return XEMA_EINVAL;
+  std::vector<xema_tensor> ts;
+  uint32_t ops = 0;
+  int rc = xema::build_trace(*cfg, m->chunks, m->axis, ts, &ops);
+  if (rc) return rc;
+  if (n_tensors) *n_tensors = ts.size();
+  if (n_ops) *n_ops = ops;
+  if (cap < ts.size() || !out) return XEMA_ENOSPC;
+  std::memcpy(out, ts.data(), ts.size() * sizeof(xema_tensor));
+  return XEMA_OK;
+}
+
+int xema_mitigation_for_budget(const xema_config* cfg, uint64_t budget_bytes, int32_t max_chunks,
+                               xema_mitigation* m, uint64_t* peak_bytes) {
+  if (!cfg || !m) return XEMA_EINVAL;
+  return xema::mitigation_for_budget(*cfg, budget_bytes, max_chunks, true, m->chunks, m->axis, peak_bytes);
 }
 
 int xema_plan_arena(const xema_tensor* tensors, size_t n, uint64_t* offsets, uint64_t* peak_bytes,

@@ -96,6 +96,7 @@ struct Op {
   int pos0;
   // shared
   int rows;
+  int batch;          // batch elements this launch covers (OP_LN, OP_ROPE)
   GemmLaunch gemm;
   AttnLaunch attn;
 };
@@ -107,6 +108,7 @@ using namespace xema;
 struct xema_plan {
   xema_config cfg;
   int32_t chunks[3];  // key/value, attention, feed-forward phase
+  int32_t axes[3];    // XEMA_SPLIT_ROWS or XEMA_SPLIT_BATCH per phase
   std::vector<xema_tensor> tensors;
   std::vector<uint64_t> offsets;
   std::unordered_map<std::string, size_t> index;
@@ -124,9 +126,9 @@ static int issue(const xema_plan* pl, const Op& op, cudaStream_t st) {
       return launch_mod(op.temb, op.w_mod, op.b_mod, op.mod, c.batch, c.temb_dim, 6 * c.hidden, st);
     case OP_LN:
       return launch_ln_modulate(op.ln_in, op.ln_in_f32, op.ln_in_batch_rows, op.ln_out, op.shift, op.scale,
-                                6LL * c.hidden, c.batch, op.rows, c.hidden, c.ln_eps, st);
+                                6LL * c.hidden, op.batch, op.rows, c.hidden, c.ln_eps, st);
     case OP_ROPE:
-      return launch_rmsnorm_rope(op.rope_x, op.rope_ld, op.rope_batch_rows, op.rope_g, pl->rope, op.pos0, c.batch,
+      return launch_rmsnorm_rope(op.rope_x, op.rope_ld, op.rope_batch_rows, op.rope_g, pl->rope, op.pos0, op.batch,
                                  op.rows, c.heads, c.head_dim, c.rms_eps, st);
     case OP_GEMM:
       return launch_gemm(op.gemm, st);
@@ -158,15 +160,29 @@ int xema_plan_create(const xema_config* cfg, int32_t chunks, xema_plan** out) {
 }
 
 int xema_plan_create_phases(const xema_config* cfg, const int32_t chunks[3], xema_plan** out) {
-  if (!cfg || !out || !chunks) return XEMA_EINVAL;
+  if (!chunks) return XEMA_EINVAL;
+  xema_mitigation m;
+  for (int i = 0; i < 3; ++i) {
+    m.chunks[i] = chunks[i];
+    m.axis[i] = XEMA_SPLIT_ROWS;
+  }
+  return xema_plan_create_mitigated(cfg, &m, out);
+}
+
+int xema_plan_create_mitigated(const xema_config* cfg, const xema_mitigation* m, xema_plan** out) {
+  if (!cfg || !out || !m) return XEMA_EINVAL;
   *out = nullptr;
   xema_plan* pl = new (std::nothrow) xema_plan();
   if (!pl) return XEMA_ENOSPC;
   pl->cfg = *cfg;
-  for (int i = 0; i < 3; ++i) pl->chunks[i] = chunks[i];
+  const int32_t* chunks = m->chunks;
+  for (int i = 0; i < 3; ++i) {
+    pl->chunks[i] = m->chunks[i];
+    pl->axes[i] = m->axis[i];
+  }
   pl->bound = false;
   pl->rope = nullptr;
-  int rc = build_trace(*cfg, chunks, pl->tensors, &pl->n_ops);
+  int rc = build_trace(*cfg, chunks, pl->axes, pl->tensors, &pl->n_ops);
   if (!rc) {
     pl->offsets.assign(pl->tensors.size(), 0);
     rc = plan_arena(pl->tensors.data(), pl->tensors.size(), pl->offsets.data(), &pl->peak, &pl->live);
@@ -196,6 +212,15 @@ int xema_plan_info(const xema_plan* plan, uint64_t* peak_bytes, uint64_t* max_li
 int xema_plan_phase_chunks(const xema_plan* plan, int32_t chunks[3]) {
   if (!plan || !chunks) return XEMA_EINVAL;
   for (int i = 0; i < 3; ++i) chunks[i] = plan->chunks[i];
+  return XEMA_OK;
+}
+
+int xema_plan_mitigation(const xema_plan* plan, xema_mitigation* m) {
+  if (!plan || !m) return XEMA_EINVAL;
+  for (int i = 0; i < 3; ++i) {
+    m->chunks[i] = plan->chunks[i];
+    m->axis[i] = plan->axes[i];
+  }
   return XEMA_OK;
 }
 
@@ -275,21 +300,48 @@ int xema_plan_bind(xema_plan* plan, void* arena_dev, uint64_t arena_bytes, const
     tag(op, "MOD", -1, 2.0 * Bd * 6 * Dd * c.temb_dim, 2.0 * 6 * Dd * c.temb_dim + 24.0 * Bd * Dd);
     plan->ops.push_back(op);
 
-    auto ln_op = [&](const void* in, int f32, void* out, int rows, int which, const char* nm, int chunk) {
+    // A piece of a phase: batch elements [b0, b0 + nb) x rows [r0, r0 + n).
+    struct Piece {
+      long long b0, r0;
+      int nb, n;
+    };
+    auto piece_of = [&](int phase, int ci) {
+      const int C = plan->chunks[phase];
+      Piece pc;
+      if (plan->axes[phase] == XEMA_SPLIT_BATCH) {
+        pc.b0 = (long long)ci * c.batch / C;
+        pc.nb = (int)((long long)(ci + 1) * c.batch / C - pc.b0);
+        pc.r0 = 0;
+        pc.n = (int)S;
+      } else {
+        pc.b0 = 0;
+        pc.nb = c.batch;
+        pc.r0 = (long long)ci * S / C;
+        pc.n = (int)((long long)(ci + 1) * S / C - pc.r0);
+      }
+      return pc;
+    };
+    // byte offset of (batch b0, row r0) in a full-size [B, S, width] tensor
+    auto at_row = [&](const Piece& pc, long long width, int elem_bytes) { return (pc.b0 * S + pc.r0) * width * elem_bytes; };
+    auto ln_op = [&](const void* in, int f32, void* out, const Piece& pc, int which, const char* nm, int chunk) {
       Op o{};
       o.kind = OP_LN;
-      tag(o, nm, chunk, 8.0 * Bd * rows * Dd, Bd * rows * Dd * (f32 ? 6.0 : 4.0));
+      const double elems = (double)pc.nb * pc.n;
+      tag(o, nm, chunk, 8.0 * elems * Dd, elems * Dd * (f32 ? 6.0 : 4.0));
       o.ln_in = in; o.ln_in_f32 = f32; o.ln_in_batch_rows = S; o.ln_out = out;
-      o.shift = mod + (which == 1 ? 0 : 3 * D);
-      o.scale = mod + (which == 1 ? D : 4 * D);
-      o.rows = rows;
+      o.shift = mod + pc.b0 * 6 * D + (which == 1 ? 0 : 3 * D);
+      o.scale = mod + pc.b0 * 6 * D + (which == 1 ? D : 4 * D);
+      o.rows = pc.n;
+      o.batch = pc.nb;
       plan->ops.push_back(o);
     };
     auto gemm_op = [&](const void* a, long long lda, long long a_batch_rows, const void* wt, long long ldw,
                        const void* bias, void* out, long long ldo, long long out_batch_rows, const void* resid,
-                       long long ldr, long long resid_batch_rows, const float* gate, int rows, int N, int K,
+                       long long ldr, long long resid_batch_rows, const float* gate, const Piece& pc, int N, int K,
                        int epi, const char* nm, int chunk, const void* norm_gain = nullptr, int norm_cols = 0,
                        int pos0 = 0) -> int {
+      const int rows = pc.n;
+      const double Bd = (double)pc.nb;
       Op o{};
       o.kind = OP_GEMM;
       o.gemm.norm_gain = norm_gain; o.gemm.rope = rope_dev; o.gemm.rope_pos0 = pos0; o.gemm.head_dim = c.head_dim;
@@ -304,76 +356,82 @@ int xema_plan_bind(xema_plan* plan, void* arena_dev, uint64_t arena_bytes, const
       g.bias = bias; g.out = out; g.ldo = ldo; g.out_batch_rows = out_batch_rows;
       g.resid = resid; g.ldr = ldr; g.resid_batch_rows = resid_batch_rows;
       g.gate = gate; g.gate_stride = 6 * D;
-      g.batch = c.batch; g.rows = rows; g.N = N; g.K = K; g.epilogue = epi; g.status = status;
+      g.batch = pc.nb; g.rows = rows; g.N = N; g.K = K; g.epilogue = epi; g.status = status;
       int rc = gemm_prepare(&g, a, lda, a_batch_rows, wt, ldw);
       if (rc) return rc;
       plan->ops.push_back(o);
       return XEMA_OK;
     };
 
-    // phase A: keys and values of every chunk
+    // phase A: keys and values of every piece
     for (int ci = 0; ci < CA; ++ci) {
-      const long long r0 = (long long)ci * S / CA, r1 = (long long)(ci + 1) * S / CA;
-      const int n = (int)(r1 - r0);
+      const Piece pc = piece_of(0, ci);
+      const int n = pc.n;
       uint8_t* h1a = at("h1a", l, ci);
       if (!h1a) return XEMA_EINVAL;
-      ln_op(hid + r0 * D * 2, 0, h1a, n, 1, "LN1A", ci);
+      uint8_t* kv_pc = kv + at_row(pc, 2 * D, 2);
+      ln_op(hid + at_row(pc, D, 2), 0, h1a, pc, 1, "LN1A", ci);
       // K half: RMSNorm * g_k + RoPE in the GEMM epilogue; the KROPE op of the trace is then
       // a placeholder (the fused kernel touches a subset of what the trace says is live)
-      int rc = gemm_op(h1a, D, n, w_qkv + D * D, D, b_qkv + D, kv + r0 * 2 * D * 2, 2 * D, S, nullptr, 0, 0, nullptr,
-                       n, (int)(2 * D), (int)D, XEMA_EPI_BIAS_NORM_ROPE, "KV", ci, w.g_k, (int)D, (int)r0);
+      int rc = gemm_op(h1a, D, n, w_qkv + D * D, D, b_qkv + D, kv_pc, 2 * D, S, nullptr, 0, 0, nullptr,
+                       pc, (int)(2 * D), (int)D, XEMA_EPI_BIAS_NORM_ROPE, "KV", ci, w.g_k, (int)D, (int)pc.r0);
       if (rc) return rc;
       Op o{};
       o.kind = OP_FUSED;
       tag(o, "KROPE", ci, 0.0, 0.0);
-      o.rope_x = kv + r0 * 2 * D * 2; o.rope_ld = 2 * D; o.rope_batch_rows = S; o.rope_g = w.g_k;
-      o.pos0 = (int)r0; o.rows = n;
+      o.rope_x = kv_pc; o.rope_ld = 2 * D; o.rope_batch_rows = S; o.rope_g = w.g_k;
+      o.pos0 = (int)pc.r0; o.rows = n; o.batch = pc.nb;
       plan->ops.push_back(o);
     }
-    // phase B: queries, attention and the gated output projection of every chunk
+    // phase B: queries, attention and the gated output projection of every piece
     for (int ci = 0; ci < CB; ++ci) {
-      const long long r0 = (long long)ci * S / CB, r1 = (long long)(ci + 1) * S / CB;
-      const int n = (int)(r1 - r0);
+      const Piece pc = piece_of(1, ci);
+      const int n = pc.n;
+      const double Bd = (double)pc.nb;
       uint8_t* h1b = at("h1b", l, ci);
       uint8_t* q = at("q", l, ci);
       uint8_t* o_t = at("o", l, ci);
       float* lse = reinterpret_cast<float*>(at("lse", l, ci));
       if (!h1b || !q || !o_t || !lse) return XEMA_EINVAL;
-      ln_op(hid + r0 * D * 2, 0, h1b, n, 1, "LN1B", ci);
-      int rc = gemm_op(h1b, D, n, w_qkv, D, b_qkv, q, D, n, nullptr, 0, 0, nullptr, n, (int)D, (int)D,
-                       XEMA_EPI_BIAS_NORM_ROPE, "Q", ci, w.g_q, (int)D, (int)r0);
+      const uint8_t* hid_pc = hid + at_row(pc, D, 2);
+      const uint8_t* kv_b = kv + pc.b0 * S * 2 * D * 2;          // keys and values of these batch elements
+      ln_op(hid_pc, 0, h1b, pc, 1, "LN1B", ci);
+      int rc = gemm_op(h1b, D, n, w_qkv, D, b_qkv, q, D, n, nullptr, 0, 0, nullptr, pc, (int)D, (int)D,
+                       XEMA_EPI_BIAS_NORM_ROPE, "Q", ci, w.g_q, (int)D, (int)pc.r0);
       if (rc) return rc;
       Op o{};
       o.kind = OP_FUSED;
       tag(o, "QROPE", ci, 0.0, 0.0);
-      o.rope_x = q; o.rope_ld = D; o.rope_batch_rows = n; o.rope_g = w.g_q; o.pos0 = (int)r0; o.rows = n;
+      o.rope_x = q; o.rope_ld = D; o.rope_batch_rows = n; o.rope_g = w.g_q; o.pos0 = (int)pc.r0; o.rows = n;
+      o.batch = pc.nb;
       plan->ops.push_back(o);
       Op a{};
       a.kind = OP_ATTN;
       // q and o once, k and v once per launch, lse
       tag(a, "ATTN", ci, 4.0 * Bd * n * Sd * Dd, 4.0 * Bd * n * Dd + 4.0 * Bd * Sd * Dd + 4.0 * Bd * c.heads * n);
-      a.attn.o = o_t; a.attn.lse = lse; a.attn.batch = c.batch; a.attn.rows = n; a.attn.keys = (int)S;
+      a.attn.o = o_t; a.attn.lse = lse; a.attn.batch = pc.nb; a.attn.rows = n; a.attn.keys = (int)S;
       a.attn.heads = c.heads; a.attn.head_dim = c.head_dim; a.attn.status = status;
-      rc = attn_prepare(&a.attn, q, D, n, kv, kv + D * 2, 2 * D, S);
+      rc = attn_prepare(&a.attn, q, D, n, kv_b, kv_b + D * 2, 2 * D, S);
       if (rc) return rc;
       plan->ops.push_back(a);
-      rc = gemm_op(o_t, D, n, w.w_o, D, w.b_o, res + r0 * D * 4, D, S, hid + r0 * D * 2, D, S, mod + 2 * D, n, (int)D,
-                   (int)D, XEMA_EPI_GATE_RES_F32, "PROJ", ci);
+      rc = gemm_op(o_t, D, n, w.w_o, D, w.b_o, res + at_row(pc, D, 4), D, S, hid_pc, D, S,
+                   mod + pc.b0 * 6 * D + 2 * D, pc, (int)D, (int)D, XEMA_EPI_GATE_RES_F32, "PROJ", ci);
       if (rc) return rc;
     }
-    // phase C: feed-forward of every chunk
+    // phase C: feed-forward of every piece
     for (int ci = 0; ci < CC; ++ci) {
-      const long long r0 = (long long)ci * S / CC, r1 = (long long)(ci + 1) * S / CC;
-      const int n = (int)(r1 - r0);
+      const Piece pc = piece_of(2, ci);
+      const int n = pc.n;
       uint8_t* h2 = at("h2", l, ci);
       uint8_t* g = at("g", l, ci);
       if (!h2 || !g) return XEMA_EINVAL;
-      ln_op(res + r0 * D * 4, 1, h2, n, 2, "LN2", ci);
-      int rc = gemm_op(h2, D, n, w.w_1, D, w.b_1, g, F, n, nullptr, 0, 0, nullptr, n, (int)F, (int)D,
+      uint8_t* res_pc = res + at_row(pc, D, 4);
+      ln_op(res_pc, 1, h2, pc, 2, "LN2", ci);
+      int rc = gemm_op(h2, D, n, w.w_1, D, w.b_1, g, F, n, nullptr, 0, 0, nullptr, pc, (int)F, (int)D,
                        XEMA_EPI_BIAS_GELU, "FFN1", ci);
       if (rc) return rc;
-      rc = gemm_op(g, F, n, w.w_2, F, w.b_2, hid_next + r0 * D * 2, D, S, res + r0 * D * 4, D, S, mod + 5 * D, n,
-                   (int)D, (int)F, XEMA_EPI_GATE_RES_BF16, "FFN2", ci);
+      rc = gemm_op(g, F, n, w.w_2, F, w.b_2, hid_next + at_row(pc, D, 2), D, S, res_pc, D, S,
+                   mod + pc.b0 * 6 * D + 5 * D, pc, (int)D, (int)F, XEMA_EPI_GATE_RES_BF16, "FFN2", ci);
       if (rc) return rc;
     }
   }

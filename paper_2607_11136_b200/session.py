@@ -24,12 +24,14 @@ class BlockSession:
               dicts name -> torch tensors already on the device.
     Either `chunks` (one count, or a triple of per-phase counts) or `budget_bytes` selects
     the chunking; with a budget, `per_phase` picks between the per-phase search (chunk only
-    the phases whose trace exceeds the budget) and one count for the whole block.
+    the phases whose trace exceeds the budget) and one count for the whole block; `serialize`
+    lets that search split a phase into sub-batches instead of row chunks where the batch allows
+    it (temporary serialization).  `axes` gives the split axis per phase for explicit `chunks`.
     """
 
     def __init__(self, template, weights: Sequence[dict], chunks=None,
                  budget_bytes: Optional[int] = None, max_chunks: int = 64, device="cuda:0",
-                 arena: Optional[torch.Tensor] = None, per_phase: bool = True):
+                 arena: Optional[torch.Tensor] = None, per_phase: bool = True, axes=None, serialize: bool = False):
         if not torch.cuda.is_available():
             raise RuntimeError("a CUDA device is required (there is no CPU fallback)")
         self.device = torch.device(device)
@@ -39,14 +41,19 @@ class BlockSession:
         if chunks is None:
             if budget_bytes is None:
                 raise ValueError("give chunks or budget_bytes")
-            search = xb.xema_phase_chunks_for_budget if per_phase else xb.xema_chunks_for_budget
-            chunks, _ = search(self.cfg, int(budget_bytes), max_chunks)
+            if serialize:
+                chunks, axes, _ = xb.xema_mitigation_for_budget(self.cfg, int(budget_bytes), max_chunks)
+                search = xb.xema_mitigation_for_budget
+            else:
+                search = xb.xema_phase_chunks_for_budget if per_phase else xb.xema_chunks_for_budget
+                chunks, _ = search(self.cfg, int(budget_bytes), max_chunks)
             if chunks is None:
                 raise xb.XemaError(xb.XEMA_EBUDGET, search.__name__)
         self.budget_bytes = budget_bytes
-        self.plan = xb.Plan(self.cfg, chunks)
+        self.plan = xb.Plan(self.cfg, chunks, axes)
         self.chunks = chunks
         self.phase_chunks = self.plan.phase_chunks
+        self.axes = self.plan.axes
         if budget_bytes is not None and self.plan.peak_bytes > budget_bytes:
             raise xb.XemaError(xb.XEMA_EBUDGET, "plan peak exceeds the budget")
         if len(weights) != template.n_blocks:

@@ -305,3 +305,49 @@ def test_pipelined_host_to_host_equals_serial(tiny_case):
             assert np.array_equal(got.numpy().view(np.uint16).reshape(exp.shape), exp)
     assert np.array_equal(want[0], _run(t, [w], x, temb, 1)[1])
     assert s.staging_bytes == 2 * x.size * 2 + temb.size * 2
+
+
+def test_sub_batch_pieces_are_bit_identical_to_row_chunks():
+    """Temporary serialization: phases split into sub-batches (whole batch elements, all rows)
+    give the bits of the unsplit block, match the oracle, and the budget search picks them."""
+    t = template("tiny", batch=3, grid_t=2)
+    w = make_block_weights(t, 4)
+    x, temb = make_activations(t)
+    ref = ob.block_forward(t, _f64(w), bits_to_f64(x), bits_to_f64(temb))
+    _, base = _run(t, [w], x, temb, 1)
+    assert_close(bits_to_f64(base), ref["y"], "batch 3 unsplit")
+    for chunks, axes in [((1, 1, 3), (0, 0, 1)), ((2, 3, 2), (1, 1, 1)), ((2, 2, 3), (0, 1, 0)), ((3, 1, 2), (1, 0, 0))]:
+        s = BlockSession(t, [w], chunks=chunks, axes=axes)
+        assert s.axes == axes and s.phase_chunks == chunks
+        s.set_inputs(x, temb)
+        s.forward()
+        assert np.array_equal(s.output_bits(), base), (chunks, axes)
+    cfg = xb.make_config(t)
+    p1 = xb.Plan(cfg, 1).peak_bytes
+    s = BlockSession(t, [w], budget_bytes=int(0.9 * p1), serialize=True)
+    # two sub-batches of three requests would still hold two of them in one piece
+    assert s.phase_chunks == (1, 1, 3) and s.axes == (0, 0, 1) and s.plan.peak_bytes <= int(0.9 * p1)
+    s.set_inputs(x, temb)
+    s.forward()
+    assert np.array_equal(s.output_bits(), base)
+
+
+def test_flux_batch_four_serialized_ffn():
+    """Flux-style block, batch 4, budget at 0.9 of the unsplit peak: the feed-forward phase runs as
+    two sub-batches of two requests; same bits as the unsplit block at sampled rows and overall."""
+    t = template("flux", batch=4)
+    w = make_block_weights(t, 0)
+    x, temb = make_activations(t)
+    cfg = xb.make_config(t)
+    p1 = xb.Plan(cfg, 1).peak_bytes
+    s1 = BlockSession(t, [w], chunks=1)
+    s1.set_inputs(x, temb)
+    s1.forward()
+    y1 = s1.output_bits()
+    dev_w = s1.weights
+    del s1
+    s = BlockSession(t, dev_w, budget_bytes=int(0.9 * p1), serialize=True)
+    assert s.phase_chunks == (1, 1, 2) and s.axes == (0, 0, 1) and s.plan.peak_bytes == s.arena.numel() <= int(0.9 * p1)
+    s.set_inputs(x, temb)
+    s.forward()
+    assert np.array_equal(s.output_bits(), y1)

@@ -129,7 +129,8 @@ def _gemm_case(rng, B, rows, N, K, epi, a_extra_rows=5):
 
 @pytest.mark.parametrize("epi", [0, 1, 2, 3])
 @pytest.mark.parametrize("B,rows,N,K", [(1, 128, 256, 64), (1, 300, 512, 512), (2, 77, 384, 192),
-                                        (1, 1000, 3072, 3072), (1, 129, 1024, 2048)])
+                                        (1, 1000, 3072, 3072), (1, 129, 1024, 2048), (3, 257, 256, 128),
+                                        (1, 5000, 768, 320)])
 def test_gemm_epilogues(epi, B, rows, N, K):
     rng = np.random.default_rng(100 + epi)
     got, ref = _gemm_case(rng, B, rows, N, K, epi)

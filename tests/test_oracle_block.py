@@ -259,3 +259,14 @@ def test_branches_are_not_negligible(tiny_out):
     assert 0.9 < rms(y) < 1.4
     assert rms(tiny_out["attn_branch"]) > 0.005
     assert rms(tiny_out["ffn_branch"]) > 0.02
+
+
+def test_sub_batch_split_equals_unchunked():
+    t = template("tiny", batch=3)
+    W = {k: bits_to_f64(v) for k, v in make_block_weights(t, 0).items()}
+    x, temb = make_activations(t)
+    x, temb = bits_to_f64(x), bits_to_f64(temb)
+    ref = ob.block_forward(t, W, x, temb)
+    for chunks, axes in [((1, 1, 3), (0, 0, 1)), ((2, 3, 2), (1, 1, 1)), ((2, 2, 3), (0, 1, 0))]:
+        out = ob.block_forward_chunked(t, W, x, temb, chunks, axes)
+        assert np.abs(out["y"] - ref["y"]).max() < 1e-12 and np.abs(out["lse"] - ref["lse"]).max() < 1e-12

@@ -345,3 +345,60 @@ def test_phase_chunks_for_budget_values():
     assert arena.phase_chunks_for_budget(template("longvideo"), 4 << 30, 8)[0] == (1, 1, 2)
     # the 42-block step: same counts as one block (the budget binds inside a block)
     assert arena.phase_chunks_for_budget(template("step"), 640 * MiB, 16)[0] == (1, 1, 2)
+
+
+# ---- temporary serialization: a phase split into sub-batches instead of row chunks -----------
+
+def test_batch_split_trace_sizes_and_lifetimes():
+    """Lifetimes do not depend on the split axis; piece sizes do: a sub-batch piece holds whole
+    batch elements (all S rows), a row chunk holds all B elements of its rows."""
+    t = template("tiny", batch=4)
+    S, D, F, H = t.seq, t.hidden, t.ffn, t.heads
+    rows, n_ops = trace.trace(t, (2, 2, 4))
+    sub, n_ops2 = trace.trace(t, (2, 2, 4), (1, 1, 1))
+    assert n_ops == n_ops2 and [(d["name"], d["birth"], d["death"]) for d in rows] == \
+        [(d["name"], d["birth"], d["death"]) for d in sub]
+    size = {d["name"]: d["bytes"] for d in sub}
+    A = trace.align_up
+    assert size["h1a0_0"] == size["q0_1"] == A(2 * 2 * S * D)          # 2 of 4 batch elements
+    assert size["lse0_0"] == A(4 * 2 * H * S)
+    assert size["g0_3"] == A(2 * 1 * S * F) and size["h20_0"] == A(2 * 1 * S * D)
+    # 3 sub-batches of 4 elements: pieces of 1, 1, 2 elements
+    sizes3 = [d["bytes"] for d in trace.trace(t, (1, 1, 3), (0, 0, 1))[0] if d["name"].startswith("g0_")]
+    assert sizes3 == [A(2 * S * F), A(2 * S * F), A(2 * 2 * S * F)]
+    # the same fraction along either axis gives the same piece size when both divide evenly
+    assert {d["name"]: d["bytes"] for d in trace.trace(t, (2, 2, 2))[0]} == \
+        {d["name"]: d["bytes"] for d in trace.trace(t, (2, 2, 2), (1, 1, 1))[0]}
+    for bad in [((5, 1, 1), (1, 0, 0)), ((1, 1, 2), (0, 0, 2))]:
+        with pytest.raises(ValueError):
+            trace.trace(t, *bad)
+    with pytest.raises(ValueError):
+        trace.trace(template("tiny"), (1, 1, 2), (0, 0, 1))             # B = 1 cannot be serialized
+
+
+def test_mitigation_for_budget_serializes_where_the_batch_allows():
+    t = template("flux", batch=4)
+    p1 = arena.plan_arena(trace.trace(t, 1)[0])[1]
+    assert arena.mitigation_for_budget(t, p1, 16) == ((1, 1, 1), (0, 0, 0), p1)
+    counts, axes, peak = arena.mitigation_for_budget(t, int(0.9 * p1), 16)
+    assert (counts, axes) == ((1, 1, 2), (0, 0, 1)) and peak == arena.phase_chunks_for_budget(t, int(0.9 * p1), 16)[1]
+    # three sub-batches of four elements still hold two elements in one piece: serialization
+    # needs four pieces where row chunking needs three
+    counts, axes, peak = arena.mitigation_for_budget(t, int(0.76 * p1), 16)
+    assert (counts, axes) == ((1, 1, 4), (0, 0, 1))
+    assert arena.phase_chunks_for_budget(t, int(0.76 * p1), 16) == ((1, 1, 3), peak)
+    # beyond B pieces the search falls back to row chunks
+    t2 = template("longvideo", batch=2)
+    p1 = arena.plan_arena(trace.trace(t2, 1)[0])[1]
+    assert arena.mitigation_for_budget(t2, int(0.9 * p1), 16)[:2] == ((1, 1, 2), (0, 0, 1))
+    assert arena.mitigation_for_budget(t2, int(0.74 * p1), 16)[:2] == ((1, 1, 3), (0, 0, 0))
+    # B = 1: identical to the per-phase search
+    t1 = template("cogvideox")
+    assert arena.mitigation_for_budget(t1, 640 << 20, 16) == ((1, 1, 2), (0, 0, 0), 600760320)
+    # every plan the search returns is valid and tight on these templates
+    for tt, frac in ((t, 0.9), (t, 0.76), (t2, 0.9)):
+        p = arena.plan_arena(trace.trace(tt, 1)[0])[1]
+        counts, axes, peak = arena.mitigation_for_budget(tt, int(frac * p), 16)
+        ts, n_ops = trace.trace(tt, counts, axes)
+        offs, pk = arena.plan_arena(ts)
+        assert pk == peak == arena.max_live_bytes(ts, n_ops) and arena.overlapping_pairs(ts, offs) == []

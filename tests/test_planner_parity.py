@@ -183,3 +183,32 @@ def test_alloc_replay_event_order_reproduces_the_live_trace():
             last = seen.get(op, last)
             got.append(last)
         assert got == live and cur == 0
+
+
+# ---- temporary serialization (sub-batch pieces) ------------------------------------------------
+
+def test_mitigated_trace_and_search_bit_exact():
+    cases = [("flux", 4), ("tiny", 3), ("longvideo", 2), ("tiny", 1), ("cogvideox", 1)]
+    for name, batch in cases:
+        t = template(name, batch=batch)
+        cfg = xb.make_config(t)
+        for counts, axes in [((1, 1, 2), (0, 0, 1)), ((2, 1, 1), (1, 0, 0)), ((1, 2, 2), (0, 1, 1)),
+                             ((2, 2, 2), (1, 1, 1)), ((3, 1, 2), (0, 0, 1)), ((1, 1, 3), (0, 0, 1)), ((2, 3, 4), (0, 0, 0))]:
+            if any(c > batch for c, a in zip(counts, axes) if a):
+                with pytest.raises(xb.XemaError) as e:
+                    xb.xema_trace_mitigated(cfg, counts, axes)
+                assert e.value.status == xb.XEMA_EINVAL
+                continue
+            want, want_ops = o_trace.trace(t, counts, axes)
+            got, got_ops = xb.xema_trace_mitigated(cfg, counts, axes)
+            assert got_ops == want_ops and got == want, (name, batch, counts, axes)
+            plan = xb.Plan(cfg, counts, axes)
+            w_offs, w_peak = o_arena.plan_arena(want)
+            assert plan.peak_bytes == w_peak and plan.axes == axes and plan.phase_chunks == counts
+            assert [d["offset"] for d in plan.tensors()] == w_offs
+        p1 = o_arena.plan_arena(o_trace.trace(t, 1)[0])[1]
+        for frac in (1.0, 0.9, 0.8, 0.76, 0.74, 0.5):
+            budget = int(p1 * frac)
+            assert xb.xema_mitigation_for_budget(cfg, budget, 16) == o_arena.mitigation_for_budget(t, budget, 16)
+    with pytest.raises(xb.XemaError):
+        xb.xema_trace_mitigated(xb.make_config(template("tiny", batch=2)), (1, 1, 2), (0, 0, 5))
