@@ -133,6 +133,15 @@ int xema_plan_arena(const xema_tensor* tensors, size_t n, uint64_t* offsets,
 int xema_chunks_for_budget(const xema_config* cfg, uint64_t budget_bytes, int32_t max_chunks,
                            int32_t* chunks, uint64_t* peak_bytes);
 
+/* The memory-pressure set (section "Applying Mitigation Only Where Needed"; planner stage
+ * "locate where memory exceeds the budget"): the maximal half-open op ranges [first, end) in
+ * which the live bytes of the trace exceed budget_bytes.  ranges (host) receives up to cap
+ * pairs (first, end) in ascending order; *n_ranges (host) always receives their number, so a
+ * call with cap = 0 sizes the array (XEMA_ENOSPC when there is at least one range).
+ * XEMA_EINVAL: a tensor with death <= birth or death > n_ops. */
+int xema_pressure_ranges(const xema_tensor* tensors, size_t n, uint32_t n_ops,
+                         uint64_t budget_bytes, uint32_t* ranges, size_t cap, size_t* n_ranges);
+
 /* Per-phase chunk counts (section "Applying Mitigation Only Where Needed": the planner
  * locates, on the memory trace, where the budget is exceeded and mitigates only there).
  * A block has three phases: 0 = keys/values (LN1A, KV, KROPE per chunk), 1 = queries,

@@ -109,6 +109,23 @@ def live_per_op(tensors, n_ops):
     return out
 
 
+def pressure_ranges(tensors, n_ops, budget_bytes):
+    """The memory-pressure set as maximal half-open op ranges [first, end) in which the
+    active-memory trace exceeds the budget (the planner's step "locate where memory exceeds the
+    budget": mitigation is applied to these ranges only)."""
+    live = live_per_op(tensors, n_ops)
+    out, start = [], None
+    for op, b in enumerate(live):
+        if b > budget_bytes and start is None:
+            start = op
+        if b <= budget_bytes and start is not None:
+            out.append((start, op))
+            start = None
+    if start is not None:
+        out.append((start, n_ops))
+    return out
+
+
 def phase_chunks_for_budget(t, budget_bytes, max_chunks):
     """Mitigation only where it is needed (the planner's stage "locating where memory exceeds
     the budget", with chunking as the mitigation): start unchunked; mark the phases in which

@@ -20,7 +20,7 @@ EPI_BIAS, EPI_BIAS_GELU, EPI_GATE_RES_F32, EPI_GATE_RES_BF16, EPI_BIAS_NORM_ROPE
 
 EXPORTS = (
     "xema_trace", "xema_trace_phases", "xema_plan_arena", "xema_chunks_for_budget",
-    "xema_phase_chunks_for_budget", "xema_trace_mitigated", "xema_mitigation_for_budget", "xema_rope_table",
+    "xema_phase_chunks_for_budget", "xema_pressure_ranges", "xema_trace_mitigated", "xema_mitigation_for_budget", "xema_rope_table",
     "xema_plan_create", "xema_plan_create_phases", "xema_plan_create_mitigated", "xema_plan_destroy",
     "xema_plan_info", "xema_plan_phase_chunks", "xema_plan_mitigation", "xema_plan_tensor",
     "xema_plan_tensor_at", "xema_plan_bind", "xema_block_forward", "xema_step_forward",
@@ -102,6 +102,7 @@ def lib() -> C.CDLL:
             "xema_plan_mitigation": [vp, P(xema_mitigation)],
             "xema_plan_phase_chunks": [vp, P(i32)],
             "xema_plan_arena": [P(xema_tensor), sz, P(u64), P(u64), P(u64)],
+            "xema_pressure_ranges": [P(xema_tensor), sz, u32, u64, P(u32), sz, P(sz)],
             "xema_pluggable_mode": [C.c_int],
             "xema_pluggable_recorded": [P(xema_tensor), sz, P(sz), P(u32)],
             "xema_pluggable_set_plan": [vp, u64, P(u64), sz],
@@ -239,6 +240,23 @@ def xema_mitigation_for_budget(cfg: xema_config, budget_bytes: int, max_chunks: 
         return None, None, peak.value
     _check(rc, "xema_mitigation_for_budget")
     return tuple(m.chunks), tuple(m.axis), peak.value
+
+
+def xema_pressure_ranges(tensors: Sequence[dict], n_ops: int, budget_bytes: int):
+    """-> list of half-open op ranges (first, end) where the live bytes exceed the budget"""
+    n = len(tensors)
+    arr = (xema_tensor * max(n, 1))()
+    for i, d in enumerate(tensors):
+        arr[i].bytes, arr[i].birth, arr[i].death = d["bytes"], d["birth"], d["death"]
+    cnt = C.c_size_t(0)
+    rc = lib().xema_pressure_ranges(arr, n, n_ops, budget_bytes, None, 0, C.byref(cnt))
+    if rc != XEMA_ENOSPC:
+        _check(rc, "xema_pressure_ranges")
+    if cnt.value == 0:
+        return []
+    out = (C.c_uint32 * (2 * cnt.value))()
+    _check(lib().xema_pressure_ranges(arr, n, n_ops, budget_bytes, out, cnt.value, C.byref(cnt)), "xema_pressure_ranges")
+    return [(out[2 * i], out[2 * i + 1]) for i in range(cnt.value)]
 
 
 def xema_plan_arena(tensors: Sequence[dict]):

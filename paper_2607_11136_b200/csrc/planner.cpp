@@ -410,6 +410,32 @@ int xema_mitigation_for_budget(const xema_config* cfg, uint64_t budget_bytes, in
   return xema::mitigation_for_budget(*cfg, budget_bytes, max_chunks, true, m->chunks, m->axis, peak_bytes);
 }
 
+int xema_pressure_ranges(const xema_tensor* tensors, size_t n, uint32_t n_ops, uint64_t budget_bytes,
+                         uint32_t* ranges, size_t cap, size_t* n_ranges) {
+  if (n && !tensors) return XEMA_EINVAL;
+  std::vector<int64_t> delta((size_t)n_ops + 1, 0);
+  for (size_t i = 0; i < n; ++i) {
+    if (tensors[i].death <= tensors[i].birth || tensors[i].death > n_ops) return XEMA_EINVAL;
+    delta[tensors[i].birth] += (int64_t)tensors[i].bytes;
+    delta[tensors[i].death] -= (int64_t)tensors[i].bytes;
+  }
+  std::vector<uint32_t> out;
+  int64_t live = 0;
+  bool open = false;
+  for (uint32_t op = 0; op < n_ops; ++op) {
+    live += delta[op];
+    const bool over = (uint64_t)live > budget_bytes;
+    if (over && !open) out.push_back(op);
+    if (!over && open) out.push_back(op);
+    open = over;
+  }
+  if (open) out.push_back(n_ops);
+  if (n_ranges) *n_ranges = out.size() / 2;
+  if (out.size() / 2 > cap || (!ranges && !out.empty())) return XEMA_ENOSPC;
+  for (size_t i = 0; i < out.size(); ++i) ranges[i] = out[i];
+  return XEMA_OK;
+}
+
 int xema_plan_arena(const xema_tensor* tensors, size_t n, uint64_t* offsets, uint64_t* peak_bytes,
                     uint64_t* max_live_bytes) {
   return xema::plan_arena(tensors, n, offsets, peak_bytes, max_live_bytes);

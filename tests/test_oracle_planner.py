@@ -402,3 +402,25 @@ def test_mitigation_for_budget_serializes_where_the_batch_allows():
         ts, n_ops = trace.trace(tt, counts, axes)
         offs, pk = arena.plan_arena(ts)
         assert pk == peak == arena.max_live_bytes(ts, n_ops) and arena.overlapping_pairs(ts, offs) == []
+
+
+def test_pressure_ranges():
+    """Where the live bytes exceed the budget, as maximal op ranges."""
+    mk = lambda size, b, e: {"bytes": size, "birth": b, "death": e}
+    ts = [mk(4, 0, 6), mk(3, 1, 3), mk(2, 2, 5), mk(5, 4, 6)]      # live per op: 4 7 9 6 11 9
+    assert arena.live_per_op(ts, 6) == [4, 7, 9, 6, 11, 9]
+    assert arena.pressure_ranges(ts, 6, 11) == []
+    assert arena.pressure_ranges(ts, 6, 8) == [(2, 3), (4, 6)]
+    assert arena.pressure_ranges(ts, 6, 6) == [(1, 3), (4, 6)]
+    assert arena.pressure_ranges(ts, 6, 3) == [(0, 6)]
+    # CogVideoX-shaped block, unchunked, 640 MiB: only the two feed-forward GEMMs are over
+    t = template("cogvideox")
+    tensors, n_ops = trace.trace(t, 1)
+    assert arena.pressure_ranges(tensors, n_ops, 640 << 20) == [(10, 12)]
+    # with the feed-forward phase in two chunks nothing is over; at 560 MiB only FFN1 of the second
+    # chunk is (the next hidden state exists by then, during the first chunk it does not)
+    tensors, n_ops = trace.trace(t, (1, 1, 2))
+    assert arena.pressure_ranges(tensors, n_ops, 640 << 20) == []
+    assert arena.pressure_ranges(tensors, n_ops, 560 << 20) == [(13, 14)]
+    # one byte below the attention peak the attention op joins the set
+    assert arena.pressure_ranges(tensors, n_ops, 549565440 - 1) == [(7, 8), (13, 14)]

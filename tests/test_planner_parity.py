@@ -212,3 +212,22 @@ def test_mitigated_trace_and_search_bit_exact():
             assert xb.xema_mitigation_for_budget(cfg, budget, 16) == o_arena.mitigation_for_budget(t, budget, 16)
     with pytest.raises(xb.XemaError):
         xb.xema_trace_mitigated(xb.make_config(template("tiny", batch=2)), (1, 1, 2), (0, 0, 5))
+
+
+def test_pressure_ranges_bit_exact():
+    rng = np.random.default_rng(3)
+    for _ in range(50):
+        n_ops = int(rng.integers(1, 12))
+        ts = []
+        for _ in range(int(rng.integers(0, 8))):
+            b = int(rng.integers(0, n_ops))
+            ts.append({"bytes": int(rng.integers(1, 9)) * 256, "birth": b, "death": int(rng.integers(b + 1, n_ops + 1))})
+        for budget in (0, 256, 1024, 2048, 1 << 20):
+            assert xb.xema_pressure_ranges(ts, n_ops, budget) == o_arena.pressure_ranges(ts, n_ops, budget)
+    for name, counts in (("cogvideox", (1, 1, 1)), ("cogvideox", (1, 1, 2)), ("step", (1, 1, 1))):
+        t = template(name)
+        ts, n_ops = o_trace.trace(t, counts)
+        for budget in (640 << 20, 560 << 20, 549565439, 1 << 40, 0):
+            assert xb.xema_pressure_ranges(ts, n_ops, budget) == o_arena.pressure_ranges(ts, n_ops, budget)
+    with pytest.raises(xb.XemaError):
+        xb.xema_pressure_ranges([{"bytes": 256, "birth": 2, "death": 2}], 4, 0)
