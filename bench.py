@@ -394,6 +394,12 @@ def main():
                 "frac": achieved / peak, "traffic": traffic, "peak_source": peaks["source"] + " (sustained)",
                 "peak_burst": peaks["bf16_burst"] if tensor_bound else None,
                 "ms_per_launch": per_launch_s * 1e3, "launches_per_step": d["launches"]}
+    if dom == "ATTN" and t.head_dim == 64 and clocks.get("sm_max_mhz"):
+        # context: with 64-wide heads there is one exponential per 4 * 64 flop and an SM retires 16 ex2 per
+        # clock; a quarter of the exponentials run as a polynomial on the FMA pipe instead
+        sms = torch.cuda.get_device_properties(dev).multi_processor_count
+        mufu = 16.0 * sms * clocks["sm_max_mhz"] * 1e6 * 4 * t.head_dim / 1e12
+        roofline["exp_rate_ceiling_tflops"] = {"all_on_mufu_at_max_clock": mufu, "three_quarters_on_mufu": mufu / 0.75}
     breakdown = {n: {"ms": round(v["ms"], 4), "share": round(v["ms"] / ms_per_step, 4),
                      "tflops": round(v["flops"] / (v["ms"] * 1e-3) / 1e12, 1) if v["ms"] > 0 else None,
                      "gbs": round(v["bytes"] / (v["ms"] * 1e-3) / 1e9, 1) if v["ms"] > 0 else None}
