@@ -262,3 +262,39 @@ def test_gemm_epilogue_rmsnorm_rope(name, norm_all):
         v = acc[b, :, :Dh].reshape(rows, H, dh)
         ref[b, :, :Dh] = ob.apply_rope(ob.rms_norm(v, gf, 1e-6), ang).reshape(rows, Dh)
     assert_bf16_close(from_dev_bf16(out), ref, ("gemm norm+rope", name, norm_all), atol_rms=3e-4)
+
+
+@pytest.mark.parametrize("dh", [64, 128])
+def test_attention_scores_growing_along_the_keys(dh):
+    """Keys whose scores rise steadily with the key index: the running max moves by more than
+    the lazy threshold again and again (every few blocks), the worst case for the rescale path;
+    and scores so far below the max that the exponentials underflow (the polynomial's clamp)."""
+    rng = np.random.default_rng(77)
+    B, rows, keys, H = 1, 200, 1100, 2
+    D = H * dh
+    u = rng.standard_normal((H, dh))
+    u /= np.linalg.norm(u, axis=1, keepdims=True)
+    ramp = np.linspace(-1.0, 1.0, keys)[:, None]
+    q = np.empty((B, rows, D)); kv = rng.standard_normal((B, keys, 2 * D))
+    for h in range(H):
+        q[0, :, h * dh:(h + 1) * dh] = u[h] * 40.0 + 0.3 * rng.standard_normal((rows, dh))
+        kv[0, :, h * dh:(h + 1) * dh] = u[h] * ramp * 60.0 + 0.3 * rng.standard_normal((keys, dh))
+    from xema_inputs import bf16_bits, bits_to_f64
+    qb, kvb = bf16_bits(q.astype(np.float32)), bf16_bits(kv.astype(np.float32))
+    qf, kvf = bits_to_f64(qb), bits_to_f64(kvb)
+    q_dev, kv_dev = to_dev(qb), to_dev(kvb)
+    o = torch.zeros(B, rows, D, dtype=torch.int16, device=DEV)
+    lse = torch.zeros(B, H, rows, dtype=torch.float32, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    xb.xema_op_attention(q_dev.data_ptr(), D, rows, kv_dev.data_ptr(), kv_dev.data_ptr() + D * 2, 2 * D, keys,
+                         o.data_ptr(), lse.data_ptr(), B, rows, keys, H, dh, status=status.data_ptr())
+    _sync_status(status)
+    got = from_dev_bf16(o)
+    for h in range(H):
+        ref_o, ref_l = ob.attention_head(qf[0, :, h * dh:(h + 1) * dh], kvf[0, :, h * dh:(h + 1) * dh],
+                                         kvf[0, :, D + h * dh:D + (h + 1) * dh], 1 / math.sqrt(dh))
+        # the scores span several hundred in the exp2 domain
+        span = (qf[0, :, h * dh:(h + 1) * dh] @ kvf[0, :, h * dh:(h + 1) * dh].T) / math.sqrt(dh) * 1.4427
+        assert span.max() - span.min() > 300
+        assert_bf16_close(got[0, :, h * dh:(h + 1) * dh], ref_o, ("growing scores", dh, h), atol_rms=2e-2, cos=0.9999)
+        assert np.abs(lse.cpu().numpy()[0, h] - ref_l).max() < 1e-3 * np.abs(ref_l).max()
