@@ -8,7 +8,7 @@ from paper_2607_11136_b200 import binding as xb
 from paper_2607_11136_b200.session import BlockSession
 from xema_inputs import bits_to_f64, make_activations, make_block_weights, sample_rows, template
 
-from gpu_util import DEV, assert_close, tolerance_split, stats
+from gpu_util import DEV, assert_bf16_close, assert_close, tolerance_split, stats
 
 pytestmark = pytest.mark.gpu
 
@@ -351,3 +351,25 @@ def test_flux_batch_four_serialized_ffn():
     s.set_inputs(x, temb)
     s.forward()
     assert np.array_equal(s.output_bits(), y1)
+
+
+def test_redundant_layer_norm_launch_is_elided_only_when_in_place(tiny_case):
+    """With one piece in the key/value and attention phases LN1B would rewrite what LN1A left at
+    the same arena address; the executor skips that launch (12 logical ops, 9 launches) and the
+    output bits do not change; with two pieces nothing is skipped."""
+    t, w, x, temb, ref = tiny_case
+    s2, y2 = _run(t, [w], x, temb, 2)
+    s1, y1 = _run(t, [w], x, temb, (1, 1, 2))
+    assert np.array_equal(y1, y2)
+    names = [s1.plan.op(i)["name"] for i in range(s1.plan.n_ops)]
+    assert names == ["MOD", "LN1A", "KV", "KROPE", "LN1B", "Q", "QROPE", "ATTN", "PROJ", "LN2", "FFN1", "FFN2", "LN2",
+                     "FFN1", "FFN2"]
+    assert s1.plan.tensor("h1a0_0") == s1.plan.tensor("h1b0_0")
+    assert s1.plan.launch_count() == 15 - 3                 # KROPE, QROPE and LN1B launch nothing
+    assert s2.plan.launch_count() == 23 - 4
+    # the intermediate the elided launch would have written is what the Q projection reads
+    s1.set_inputs(x, temb)
+    s1.plan.forward_prefix(5, torch.cuda.current_stream().cuda_stream)      # up to and including LN1B
+    torch.cuda.synchronize()
+    h1 = s1.view("h1b0_0", torch.int16, (1, t.seq, t.hidden)).cpu().numpy().view(np.uint16)
+    assert_bf16_close(bits_to_f64(h1), ref["h1"], "h1 left in place by LN1A")
