@@ -111,6 +111,21 @@ class BlockSession:
         else:
             self.plan.step_forward(s)
 
+    def capture(self, stream: Optional[torch.cuda.Stream] = None) -> "torch.cuda.CUDAGraph":
+        """Records one forward pass into a CUDA graph (every address is static, so the graph
+        stays valid for as long as the session lives); `graph.replay()` then costs one launch on
+        the host instead of one per kernel.  The first call warms the kernels up eagerly."""
+        st = stream or torch.cuda.Stream(self.device)
+        st.wait_stream(torch.cuda.current_stream(self.device))
+        with torch.cuda.stream(st):
+            self.forward(st)                      # one-time function attributes are set outside capture
+        st.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=st):
+            self.forward(st)
+        torch.cuda.current_stream(self.device).wait_stream(st)
+        return g
+
     def output_bits(self) -> np.ndarray:
         """Synchronises and returns the output hidden state as uint16 bf16 bit patterns."""
         out = self.hid_out().cpu().numpy().view(np.uint16)

@@ -373,3 +373,29 @@ def test_redundant_layer_norm_launch_is_elided_only_when_in_place(tiny_case):
     torch.cuda.synchronize()
     h1 = s1.view("h1b0_0", torch.int16, (1, t.seq, t.hidden)).cpu().numpy().view(np.uint16)
     assert_bf16_close(bits_to_f64(h1), ref["h1"], "h1 left in place by LN1A")
+
+
+def test_forward_replayed_from_a_cuda_graph(tiny_case):
+    """A captured forward pass replays to the same bits as the eager one (every address is static)."""
+    t, w, x, temb, ref = tiny_case
+    s, want = _run(t, [w], x, temb, (1, 1, 2))
+    g = s.capture()
+    for _ in range(3):
+        s.set_inputs(x, temb)
+        s.hid_out().zero_()
+        g.replay()
+        assert np.array_equal(s.output_bits(), want)
+    import time
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(200):
+        g.replay()
+    torch.cuda.synchronize()
+    t_graph = (time.perf_counter() - t0) / 200
+    t0 = time.perf_counter()
+    for _ in range(200):
+        s.forward()
+    torch.cuda.synchronize()
+    t_eager = (time.perf_counter() - t0) / 200
+    print("tiny block: %.1f us per replayed graph, %.1f us eager" % (t_graph * 1e6, t_eager * 1e6))
+    s.check_status()
