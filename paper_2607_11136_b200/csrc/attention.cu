@@ -296,14 +296,14 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       // p = exp2(s * c - m * c) on pairs of columns with packed fp32x2 arithmetic; POLY_NUM of
       // every POLY_DEN pairs (fixed column positions) evaluate 2^x as a polynomial on the FMA
       // pipe, the rest on the MUFU; row sum in four independent packed partial sums
-      const uint64_t c2 = pack_f32x2(p.scale_log2, p.scale_log2);
-      const uint64_t nm2 = pack_f32x2(neg_m, neg_m);
-      uint64_t ls2[4] = {0ull, 0ull, 0ull, 0ull};
+      const f32x2 c2 = pack_f32x2(p.scale_log2, p.scale_log2);
+      const f32x2 nm2 = pack_f32x2(neg_m, neg_m);
+      f32x2 ls2[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
       uint32_t pk[ATT_BN / 2];
 #pragma unroll
       for (int t = 0; t < ATT_BN; t += 2) {
         const int pair = t >> 1;
-        uint64_t e2 = fma_f32x2(pack_f32x2(s[t], s[t + 1]), c2, nm2);
+        f32x2 e2 = fma_f32x2(pack_f32x2(s[t], s[t + 1]), c2, nm2);
         float e0, e1;
         if ((pair % POLY_DEN) < POLY_NUM) {
           e2 = exp2_poly_f32x2(e2);

@@ -360,67 +360,34 @@ __device__ __forceinline__ float ex2_approx(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
-// ---- packed fp32x2 arithmetic (two floats in one 64-bit register pair) ---------------------
-__device__ __forceinline__ uint64_t pack_f32x2(float lo, float hi) {
-  uint64_t r;
-  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-  return r;
+// ---- packed fp32x2 arithmetic (two floats in one register pair, one instruction for both) -----
+// Built on the compiler's float2 intrinsics so that register pairs are allocated by the compiler
+// (opaque inline assembly forced extra register moves around every packed operation).
+typedef float2 f32x2;
+__device__ __forceinline__ f32x2 pack_f32x2(float lo, float hi) { return make_float2(lo, hi); }
+__device__ __forceinline__ void unpack_f32x2(f32x2 v, float& lo, float& hi) {
+  lo = v.x;
+  hi = v.y;
 }
-__device__ __forceinline__ void unpack_f32x2(uint64_t v, float& lo, float& hi) {
-  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
-}
-__device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c) {
-  uint64_t d;
-  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-  return d;
-}
-__device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b) {
-  uint64_t d;
-  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-  return d;
-}
+__device__ __forceinline__ f32x2 fma_f32x2(f32x2 a, f32x2 b, f32x2 c) { return __ffma2_rn(a, b, c); }
+__device__ __forceinline__ f32x2 add_f32x2(f32x2 a, f32x2 b) { return __fadd2_rn(a, b); }
 // 2^x for two values on the FMA pipe instead of the MUFU: round-to-nearest split x = n + r with
 // |r| <= 1/2 through the 1.5 * 2^23 trick, a cubic for 2^r (relative error 7.5e-5, far below the
 // bf16 rounding of the probabilities it feeds), then n added into the exponent field.
 // Valid for x <= 126; inputs below -125 are clamped (2^-125 stands in for zero).
-__device__ __forceinline__ uint64_t exp2_poly_f32x2(uint64_t x2) {
-  float x0, x1;
-  unpack_f32x2(x2, x0, x1);
-  x2 = pack_f32x2(fmaxf(x0, -125.f), fmaxf(x1, -125.f));
-  const uint64_t magic = pack_f32x2(12582912.f, 12582912.f);
-  const uint64_t neg_magic = pack_f32x2(-12582912.f, -12582912.f);
-  const uint64_t neg_one = pack_f32x2(-1.f, -1.f);
-  const uint64_t t2 = add_f32x2(x2, magic);                 // integer part lands in the low mantissa bits
-  const uint64_t n2 = add_f32x2(t2, neg_magic);             // nearest integer as a float
-  const uint64_t r2 = fma_f32x2(n2, neg_one, x2);           // r = x - n
-  uint64_t p2 = fma_f32x2(pack_f32x2(0.0551716685f, 0.0551716685f), r2, pack_f32x2(0.242611125f, 0.242611125f));
-  p2 = fma_f32x2(p2, r2, pack_f32x2(0.693260968f, 0.693260968f));
-  p2 = fma_f32x2(p2, r2, pack_f32x2(0.999928057f, 0.999928057f));
-  float t0, t1, p0, p1;
-  unpack_f32x2(t2, t0, t1);
-  unpack_f32x2(p2, p0, p1);
-  const float e0 = __uint_as_float(__float_as_uint(p0) + (__float_as_uint(t0) << 23));
-  const float e1 = __uint_as_float(__float_as_uint(p1) + (__float_as_uint(t1) << 23));
-  return pack_f32x2(e0, e1);
-}
-
-// Same polynomial for a pair whose inputs are already >= -125; results come back unpacked
-// (the caller packs them to bf16 and adds them to its row sum).
-__device__ __forceinline__ void exp2_poly_pair(uint64_t x2, float& e0, float& e1) {
-  const uint64_t magic = pack_f32x2(12582912.f, 12582912.f);
-  const uint64_t neg_magic = pack_f32x2(-12582912.f, -12582912.f);
-  const uint64_t neg_one = pack_f32x2(-1.f, -1.f);
-  const uint64_t t2 = add_f32x2(x2, magic);
-  const uint64_t n2 = add_f32x2(t2, neg_magic);
-  const uint64_t r2 = fma_f32x2(n2, neg_one, x2);
-  uint64_t p2 = fma_f32x2(pack_f32x2(0.0551716685f, 0.0551716685f), r2, pack_f32x2(0.242611125f, 0.242611125f));
-  p2 = fma_f32x2(p2, r2, pack_f32x2(0.693260968f, 0.693260968f));
-  p2 = fma_f32x2(p2, r2, pack_f32x2(0.999928057f, 0.999928057f));
-  float t0, t1, p0, p1;
-  unpack_f32x2(t2, t0, t1);
-  unpack_f32x2(p2, p0, p1);
-  e0 = __uint_as_float(__float_as_uint(p0) + (__float_as_uint(t0) << 23));
-  e1 = __uint_as_float(__float_as_uint(p1) + (__float_as_uint(t1) << 23));
+__device__ __forceinline__ f32x2 exp2_poly_f32x2(f32x2 x2) {
+  x2 = make_float2(fmaxf(x2.x, -125.f), fmaxf(x2.y, -125.f));
+  const f32x2 magic = make_float2(12582912.f, 12582912.f);
+  const f32x2 neg_magic = make_float2(-12582912.f, -12582912.f);
+  const f32x2 neg_one = make_float2(-1.f, -1.f);
+  const f32x2 t2 = add_f32x2(x2, magic);                 // integer part lands in the low mantissa bits
+  const f32x2 n2 = add_f32x2(t2, neg_magic);             // nearest integer as a float
+  const f32x2 r2 = fma_f32x2(n2, neg_one, x2);           // r = x - n
+  f32x2 p2 = fma_f32x2(make_float2(0.0551716685f, 0.0551716685f), r2, make_float2(0.242611125f, 0.242611125f));
+  p2 = fma_f32x2(p2, r2, make_float2(0.693260968f, 0.693260968f));
+  p2 = fma_f32x2(p2, r2, make_float2(0.999928057f, 0.999928057f));
+  return make_float2(__uint_as_float(__float_as_uint(p2.x) + (__float_as_uint(t2.x) << 23)),
+                     __uint_as_float(__float_as_uint(p2.y) + (__float_as_uint(t2.y) << 23)));
 }
 
 // max of three values in one instruction
