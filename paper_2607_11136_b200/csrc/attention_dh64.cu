@@ -90,7 +90,7 @@ attention_dh64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
     }
     for (int t = 0; t < TILES; ++t) {
       mbar_init(&s_full[t], 1);
-      mbar_init(&p_full[t], 4);
+      mbar_init(&p_full[t], 128);   // every softmax thread of the tile arrives (no divergent single-lane arrive)
       mbar_init(&pv_done[t], 1);
     }
     *abort_flag = 0;
@@ -301,8 +301,7 @@ attention_dh64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
       tmem_st32(s_tmem, pk);
       tmem_st_wait();
       tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&p_full[tile]);
+      mbar_arrive(&p_full[tile]);
     }
     if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&pv_done[tile], (uint32_t)(n_kv - 1) & 1u, abort_flag));
     if (ok) {
