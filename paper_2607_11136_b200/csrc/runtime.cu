@@ -412,7 +412,11 @@ int xema_plan_bind(xema_plan* plan, void* arena_dev, uint64_t arena_bytes, const
           const bool overlaps = plan->offsets[i] < plan->offsets[ia] + ta.bytes && plan->offsets[ia] < plan->offsets[i] + tt.bytes;
           if (born_between && overlaps) untouched = false;
         }
-        if (untouched && ta.bytes == tb.bytes) plan->ops.back().kind = OP_FUSED;
+        if (untouched && ta.bytes == tb.bytes) {
+          plan->ops.back().kind = OP_FUSED;
+          plan->ops.back().flops = 0.0;
+          plan->ops.back().bytes = 0.0;
+        }
       }
       int rc = gemm_op(h1b, D, n, w_qkv, D, b_qkv, q, D, n, nullptr, 0, 0, nullptr, pc, (int)D, (int)D,
                        XEMA_EPI_BIAS_NORM_ROPE, "Q", ci, w.g_q, (int)D, (int)pc.r0);
