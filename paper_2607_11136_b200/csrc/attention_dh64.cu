@@ -241,58 +241,45 @@ attention_dh64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
         mx[u] = fmaxf(mx[u], s[16 * u + 15]);
       }
       const float m_blk = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+      // the running max moves only when it grows by more than 2^8 (exp2 domain); per row
+      float m_new = m_run;
+      if (j == 0 || (m_blk - m_run) * p.scale_log2 > 8.f) m_new = m_blk;
+      const float alpha = (j == 0 || m_new == m_run) ? 1.f : ex2_approx((m_run - m_new) * p.scale_log2);
+      const float neg_m = -m_new * p.scale_log2;
       // p = exp2(s * c - m * c) on pairs of columns with packed fp32x2 arithmetic; POLY_NUM of
       // every POLY_DEN pairs (fixed column positions) evaluate 2^x as a polynomial on the FMA
       // pipe, the rest on the MUFU; row sum in four independent packed partial sums
       const f32x2 c2 = pack_f32x2(p.scale_log2, p.scale_log2);
+      const f32x2 nm2 = pack_f32x2(neg_m, neg_m);
+      f32x2 ls2[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
       uint32_t pk[BN / 2];
-      auto probabilities = [&](float neg_m) -> float {
-        const f32x2 nm2 = pack_f32x2(neg_m, neg_m);
-        f32x2 ls2[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
 #pragma unroll
-        for (int t = 0; t < BN; t += 2) {
-          const int pair = t >> 1;
-          f32x2 e2 = fma_f32x2(pack_f32x2(s[t], s[t + 1]), c2, nm2);
-          float e0, e1;
-          if ((pair % POLY_DEN) < POLY_NUM) {
-            e2 = exp2_poly_f32x2(e2);
-            unpack_f32x2(e2, e0, e1);
-          } else {
-            unpack_f32x2(e2, e0, e1);
-            e0 = ex2_approx(e0);
-            e1 = ex2_approx(e1);
-            e2 = pack_f32x2(e0, e1);
-          }
-          ls2[pair & 3] = add_f32x2(ls2[pair & 3], e2);
-          pk[pair] = pack_bf16x2(e0, e1);
+      for (int t = 0; t < BN; t += 2) {
+        const int pair = t >> 1;
+        f32x2 e2 = fma_f32x2(pack_f32x2(s[t], s[t + 1]), c2, nm2);
+        float e0, e1;
+        if ((pair % POLY_DEN) < POLY_NUM) {
+          e2 = exp2_poly_f32x2(e2);
+          unpack_f32x2(e2, e0, e1);
+        } else {
+          unpack_f32x2(e2, e0, e1);
+          e0 = ex2_approx(e0);
+          e1 = ex2_approx(e1);
+          e2 = pack_f32x2(e0, e1);
         }
-        return ((ls2[0].x + ls2[0].y) + (ls2[1].x + ls2[1].y)) + ((ls2[2].x + ls2[2].y) + (ls2[3].x + ls2[3].y));
-      };
-      // The running max moves only when it grows by more than 2^8 (exp2 domain), per row -- rare
-      // after the first block.  So the probabilities are formed against the running max right
-      // away, with the block max computed beside them instead of in front of them; if a row's
-      // max does move (any row of the warp), the scores are read again and the block is redone
-      // with the new max.  Rows that keep their max get the same values either way.
-      float l_blk = probabilities(-m_run * p.scale_log2);
-      const bool moved = (j == 0) || (m_blk - m_run) * p.scale_log2 > 8.f;
-      float m_new = m_run, alpha = 1.f;
-      if (__any_sync(0xffffffffu, moved)) {
-#pragma unroll
-        for (int ch = 0; ch < BN / 32; ++ch)
-          tmem_ld32(s_tmem + ch * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[ch * 32]));
-        tmem_ld_wait();
-        if (valid < BN) {
-#pragma unroll
-          for (int t = 0; t < BN; ++t)
-            if (t >= valid) s[t] = -INFINITY;
-        }
-        if (moved) {
-          m_new = m_blk;
-          if (j > 0) alpha = ex2_approx((m_run - m_new) * p.scale_log2);
-        }
-        l_blk = probabilities(-m_new * p.scale_log2);
+        ls2[pair & 3] = add_f32x2(ls2[pair & 3], e2);
+        pk[pair] = pack_bf16x2(e0, e1);
       }
-      l_run = fmaf(l_run, alpha, l_blk);
+      float ls[4];
+      {
+        float a0, a1;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          unpack_f32x2(ls2[u], a0, a1);
+          ls[u] = a0 + a1;
+        }
+      }
+      l_run = fmaf(l_run, alpha, (ls[0] + ls[1]) + (ls[2] + ls[3]));
       m_run = m_new;
       // rescale O where the max moved (rows that kept their max multiply by exactly 1); only
       // then must PV(j-1) have finished
