@@ -50,3 +50,15 @@ def test_single_process_needs_no_group():
     t = template("cogvideox")
     assert abs(bench.block_flops(t) - 7.910e12) / 7.910e12 < 1e-3
     assert bench.attention_traffic_bytes(t, 2222) == 254.4e6
+
+
+def test_reference_arm_runs_on_rank_zero_only():
+    """Under torchrun the reference arm is printed by rank 0 alone; every other rank exits 0
+    without output and without work."""
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = dict(os.environ, RANK="1", LOCAL_RANK="1", WORLD_SIZE="2", MASTER_ADDR="127.0.0.1", MASTER_PORT=str(_free_port()))
+    r = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--impl", "reference", "--gpus", "2",
+                        "--steps", "1", "--warmup", "3"], env=env, capture_output=True, text=True, timeout=120)
+    assert r.returncode == 0 and r.stdout.strip() == ""
