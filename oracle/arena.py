@@ -76,17 +76,6 @@ def overlapping_pairs(tensors, offsets):
     return bad
 
 
-def reserved_per_op(tensors, offsets, n_ops):
-    """Reserved-memory trace: for every op, the highest address used by a tensor live at it."""
-    out = [0] * n_ops
-    for d, off in zip(tensors, offsets):
-        top = off + d["bytes"]
-        for op in range(d["birth"], d["death"]):
-            if top > out[op]:
-                out[op] = top
-    return out
-
-
 def phase_of_op(t, counts, op):
     """0 / 1 / 2 for an op of the key-value / attention / feed-forward phase of its block; the
     MOD op belongs to phase 0."""

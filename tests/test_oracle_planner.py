@@ -42,6 +42,42 @@ def test_algorithm1_worked_examples(ex):
     assert arena.overlapping_pairs(ex["tensors"], offsets) == []
 
 
+def test_overlap_checker_reports_hand_made_collisions():
+    """Negative control for the validity checker behind every "no overlaps" assertion: layouts
+    written by hand with known collisions must come back with exactly the offending pairs."""
+    ts = [_mk(1024, 0, 4), _mk(512, 0, 2), _mk(512, 1, 4), _mk(256, 2, 4)]
+    good = [0, 1024, 1536, 1024]                 # worked example (i): D reuses B's hole
+    assert arena.overlapping_pairs(ts, good) == []
+    # D moved up to 1536: it now shares [1536, 1792) with C, which is live with it
+    assert arena.overlapping_pairs(ts, [0, 1024, 1536, 1536]) == [(2, 3)]
+    # B placed inside A while both are live; C one byte into A's last byte; D alone is fine
+    assert arena.overlapping_pairs(ts, [0, 512, 1023, 2048]) == [(0, 1), (0, 2), (1, 2)]
+    # same addresses, lifetimes that only touch ([0,2) then [2,4)) are no collision ...
+    assert arena.overlapping_pairs([_mk(512, 0, 2), _mk(512, 2, 4)], [0, 0]) == []
+    # ... one op of common life is
+    assert arena.overlapping_pairs([_mk(512, 0, 3), _mk(512, 2, 4)], [0, 0]) == [(0, 1)]
+    # address ranges that only touch ([0,512) and [512,768)) are no collision; one byte less is
+    assert arena.overlapping_pairs([_mk(512, 0, 3), _mk(256, 0, 3)], [0, 512]) == []
+    assert arena.overlapping_pairs([_mk(512, 0, 3), _mk(256, 0, 3)], [0, 511]) == [(0, 1)]
+    # a tensor wholly inside another, and the order of the pair does not matter
+    assert arena.overlapping_pairs([_mk(256, 1, 2), _mk(2048, 0, 5)], [512, 0]) == [(0, 1)]
+    # a corrupted Algorithm 1 result is caught: shift one offset of a real plan onto a neighbour
+    t = template("tiny")
+    tensors, _ = trace.trace(t, 2)
+    offsets, _ = arena.plan_arena(tensors)
+    assert arena.overlapping_pairs(tensors, offsets) == []
+    hit = 0
+    for i in range(len(tensors)):
+        for j in range(len(tensors)):
+            if i != j and arena.conflicts(tensors[i], tensors[j]):
+                moved = list(offsets)
+                moved[i] = offsets[j]
+                pairs = arena.overlapping_pairs(tensors, moved)
+                assert (min(i, j), max(i, j)) in pairs
+                hit += 1
+    assert hit > 50
+
+
 def _optimal_peak(tensors):
     """Brute force: every placement order with lowest-address first-fit.  For interval
     conflict graphs this reaches the optimum on the tiny cases used here."""
