@@ -245,6 +245,8 @@ def main():
     ap.add_argument("--cpu-rows", type=int, default=CPU_SAMPLE_ROWS)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep", action="store_true", help="also time chunk counts 1, 2, 4, 8 (outside the timed region)")
+    ap.add_argument("--sustained-seconds", type=float, default=3.0,
+                    help="length of the extra sustained leg (after 2 s of pre-heat); 0 skips it")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
@@ -297,39 +299,61 @@ def main():
         torch.cuda.synchronize(dev)
 
     # ---- device-resident timing: K steps, per-op events on the launching stream ---------------
+    def timed_steps(n_steps):
+        """n_steps steps, each restoring the inputs and issuing every op, with an event between
+        ops; clocks sampled meanwhile.  Returns (total ms, sorted per-step ms, restore ms, per-op
+        dict, clocks)."""
+        sampler = ClockSampler(local)
+        sampler.start()
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(n_launch + 1)] for _ in range(n_steps)]
+        ev_in = [torch.cuda.Event(enable_timing=True) for _ in range(n_steps)]
+        barrier()
+        for k in range(n_steps):
+            ev_in[k].record(stream)
+            sess.set_inputs(x_dev, temb_dev, non_blocking=True)
+            for i in range(n_launch):
+                ev[k][i].record(stream)
+                sess.plan.forward_range(i, i + 1, stream.cuda_stream)
+            ev[k][n_launch].record(stream)
+        barrier()
+        clk = sampler.stop()
+        total = ev_in[0].elapsed_time(ev[-1][n_launch])
+        steps_sorted = sorted(ev_in[k].elapsed_time(ev[k][n_launch]) for k in range(n_steps))
+        restore = sum(ev_in[k].elapsed_time(ev[k][0]) for k in range(n_steps)) / n_steps
+        ops_t = {}
+        for i, op in enumerate(ops):
+            d = ops_t.setdefault(op["name"], {"ms": 0.0, "flops": 0.0, "bytes": 0.0, "launches": 0})
+            d["ms"] += sum(ev[k][i].elapsed_time(ev[k][i + 1]) for k in range(n_steps)) / n_steps
+            d["flops"] += op["flops"]; d["bytes"] += op["bytes"]; d["launches"] += 1
+        return total, steps_sorted, restore, ops_t, clk
+
     for _ in range(args.warmup):
         sess.set_inputs(x_dev, temb_dev, non_blocking=True)
         sess.forward(stream)
     barrier()
     free_before, _ = torch.cuda.mem_get_info(dev)
-    sampler = ClockSampler(local)
-    sampler.start()
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(n_launch + 1)] for _ in range(args.steps)]
-    ev_in = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
-    barrier()
-    for k in range(args.steps):
-        ev_in[k].record(stream)
-        sess.set_inputs(x_dev, temb_dev, non_blocking=True)
-        for i in range(n_launch):
-            ev[k][i].record(stream)
-            sess.plan.forward_range(i, i + 1, stream.cuda_stream)
-        ev[k][n_launch].record(stream)
-    barrier()
-    clocks = sampler.stop()
+    total_ms, step_ms, restore_ms, per_op, clocks = timed_steps(args.steps)
     free_after, _ = torch.cuda.mem_get_info(dev)
     sess.check_status()
-    total_ms = max_over_ranks(ev_in[0].elapsed_time(ev[-1][n_launch]), dist, dev)
+    total_ms = max_over_ranks(total_ms, dist, dev)
     ms_per_step = total_ms / args.steps
-    step_ms = sorted(ev_in[k].elapsed_time(ev[k][n_launch]) for k in range(args.steps))
-    restore_ms = sum(ev_in[k].elapsed_time(ev[k][0]) for k in range(args.steps)) / args.steps
     out_finite = bool(torch.isfinite(sess.hid_out().view(torch.bfloat16).float()).all().item())
     value = whole_job_tflops(flops, world, ms_per_step)
 
-    per_op = {}
-    for i, op in enumerate(ops):
-        d = per_op.setdefault(op["name"], {"ms": 0.0, "flops": 0.0, "bytes": 0.0, "launches": 0})
-        d["ms"] += sum(ev[k][i].elapsed_time(ev[k][i + 1]) for k in range(args.steps)) / args.steps
-        d["flops"] += op["flops"]; d["bytes"] += op["bytes"]; d["launches"] += 1
+    # ---- sustained leg: the same loop after a pre-heat, long enough for the power governor --------
+    sustained = None
+    if args.sustained_seconds > 0:
+        est = max(ms_per_step, 1e-3)
+        for _ in range(max(1, int(2000.0 / est))):            # about 2 s of pre-heat, untimed
+            sess.set_inputs(x_dev, temb_dev, non_blocking=True)
+            sess.forward(stream)
+        n_sus = max(3, int(args.sustained_seconds * 1000.0 / est))
+        s_total, s_steps, _, s_ops, s_clk = timed_steps(n_sus)
+        sess.check_status()
+        s_total = max_over_ranks(s_total, dist, dev)
+        sustained = {"steps": n_sus, "preheat_seconds": 2.0, "ms_per_step": s_total / n_sus,
+                     "ms_median": s_steps[len(s_steps) // 2], "value": whole_job_tflops(flops, world, s_total / n_sus),
+                     "clocks": s_clk, "per_op_raw": s_ops}
 
     # ---- end to end through the public API: pinned host -> arena, forward, output -> host ------
     x_host = torch.from_numpy(x_bits.view(np.int16)).pin_memory()
@@ -338,9 +362,8 @@ def main():
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
 
     def e2e_step():
-        sess.set_inputs(x_host, temb_host, non_blocking=True)
-        sess.forward(stream)
-        out_host.copy_(sess.hid_out(), non_blocking=True)
+        # the C ABI's host-buffer call: both copies and every launch on this stream, arena only
+        sess.plan.forward_host(x_host.data_ptr(), temb_host.data_ptr(), out_host.data_ptr(), stream.cuda_stream)
 
     for _ in range(3):
         e2e_step()
@@ -394,35 +417,70 @@ def main():
 
     # ---- roofline of the dominant kernel ---------------------------------------------------------
     peaks = load_peaks()
-    dom = max(per_op, key=lambda n: per_op[n]["ms"])
-    d = per_op[dom]
-    per_launch_s = d["ms"] * 1e-3 / d["launches"]
-    tensor_bound = dom in ("KV", "Q", "ATTN", "PROJ", "FFN1", "FFN2")
-    if tensor_bound:
-        achieved = d["flops"] / d["launches"] / per_launch_s / 1e12
-        peak, unit, bound = peaks["bf16_sustained"], "TFLOP/s", "tensor"
-    else:
-        achieved = d["bytes"] / d["launches"] / per_launch_s / 1e9
-        peak, unit, bound = peaks["hbm_gbs"], "GB/s", "hbm"
-    traffic = None
-    if dom == "ATTN":
-        traffic = attention_traffic_bytes(t, t.seq * t.n_blocks // d["launches"])
-    roofline = {"kernel": dom, "bound": bound, "achieved": achieved, "peak": peak, "unit": unit,
-                "frac": achieved / peak, "traffic": traffic, "peak_source": peaks["source"] + " (sustained)",
-                "peak_burst": peaks["bf16_burst"] if tensor_bound else None,
-                "ms_per_launch": per_launch_s * 1e3, "launches_per_step": d["launches"]}
+    TENSOR_OPS = ("KV", "Q", "ATTN", "PROJ", "FFN1", "FFN2")
+
+    def regime_of(clk):
+        """A kernel timed while the SM clock holds within 5 % of its maximum is compared with the
+        burst peak; one timed under the power cap with the sustained peak."""
+        if clk.get("sm_mhz") and clk.get("sm_max_mhz") and clk["sm_mhz"] >= 0.95 * clk["sm_max_mhz"]:
+            return "burst"
+        return "sustained"
+
+    def roofline_of(ops_t, clk):
+        dom = max(ops_t, key=lambda n: ops_t[n]["ms"])
+        d = ops_t[dom]
+        per_launch_s = d["ms"] * 1e-3 / d["launches"]
+        regime = regime_of(clk)
+        if dom in TENSOR_OPS:
+            achieved = d["flops"] / d["launches"] / per_launch_s / 1e12
+            peak = peaks["bf16_burst"] if regime == "burst" else peaks["bf16_sustained"]
+            unit, bound = "TFLOP/s", "tensor"
+        else:
+            achieved = d["bytes"] / d["launches"] / per_launch_s / 1e9
+            peak, unit, bound = peaks["hbm_gbs"], "GB/s", "hbm"
+        r = {"kernel": dom, "bound": bound, "achieved": achieved, "peak": peak, "unit": unit, "frac": achieved / peak,
+             "peak_source": "%s (%s: median SM clock %s of %s MHz)" % (peaks["source"], regime if bound == "tensor" else "copy",
+                                                                      clk.get("sm_mhz"), clk.get("sm_max_mhz")),
+             "ms_per_launch": per_launch_s * 1e3, "launches_per_step": d["launches"]}
+        if bound == "tensor":
+            r["frac_of_burst"] = achieved / peaks["bf16_burst"]
+            r["frac_of_sustained"] = achieved / peaks["bf16_sustained"]
+            r["frac_of_nominal_2250"] = achieved / 2250.0
+            r["peak_burst"], r["peak_sustained"] = peaks["bf16_burst"], peaks["bf16_sustained"]
+        r["traffic"] = None
+        if dom == "ATTN":
+            r["traffic"] = attention_traffic_bytes(t, t.seq * t.n_blocks // d["launches"])
+            r["traffic_source"] = ("not measured in this run: dram__bytes_read.sum + dram__bytes_write.sum of one ncu "
+                                   "capture, see profiles/attention_dh64_*.md" if r["traffic"] else None)
+        return r
+
+    def breakdown_of(ops_t, step_ms_):
+        return {n: {"ms": round(v["ms"], 4), "share": round(v["ms"] / step_ms_, 4),
+                    "tflops": round(v["flops"] / (v["ms"] * 1e-3) / 1e12, 1) if v["ms"] > 0 else None,
+                    "gbs": round(v["bytes"] / (v["ms"] * 1e-3) / 1e9, 1) if v["ms"] > 0 else None}
+                for n, v in ops_t.items()}
+
+    def tensor_ops_of(ops_t):
+        ms = sum(v["ms"] for n, v in ops_t.items() if n in TENSOR_OPS)
+        fl = sum(v["flops"] for n, v in ops_t.items() if n in TENSOR_OPS)
+        tf = fl / (ms * 1e-3) / 1e12
+        return {"tflops": tf, "ms": ms, "frac_of_burst": tf / peaks["bf16_burst"],
+                "frac_of_sustained": tf / peaks["bf16_sustained"], "frac_of_nominal_2250": tf / 2250.0}
+
+    roofline = roofline_of(per_op, clocks)
+    dom = roofline["kernel"]
     if dom == "ATTN" and t.head_dim == 64 and clocks.get("sm_max_mhz"):
         # context: with 64-wide heads there is one exponential per 4 * 64 flop and an SM retires 16 ex2 per
-        # clock; a quarter of the exponentials run as a polynomial on the FMA pipe instead
+        # clock; three eighths of the exponentials run as a polynomial on the FMA pipe instead
         sms = torch.cuda.get_device_properties(dev).multi_processor_count
         mufu = 16.0 * sms * clocks["sm_max_mhz"] * 1e6 * 4 * t.head_dim / 1e12
-        roofline["exp_rate_ceiling_tflops"] = {"all_on_mufu_at_max_clock": mufu, "three_quarters_on_mufu": mufu / 0.75}
-    breakdown = {n: {"ms": round(v["ms"], 4), "share": round(v["ms"] / ms_per_step, 4),
-                     "tflops": round(v["flops"] / (v["ms"] * 1e-3) / 1e12, 1) if v["ms"] > 0 else None,
-                     "gbs": round(v["bytes"] / (v["ms"] * 1e-3) / 1e9, 1) if v["ms"] > 0 else None}
-                 for n, v in per_op.items()}
-    tensor_ms = sum(v["ms"] for n, v in per_op.items() if n in ("KV", "Q", "ATTN", "PROJ", "FFN1", "FFN2"))
-    tensor_fl = sum(v["flops"] for n, v in per_op.items() if n in ("KV", "Q", "ATTN", "PROJ", "FFN1", "FFN2"))
+        roofline["exp_rate_ceiling_tflops"] = {"all_on_mufu_at_max_clock": mufu, "five_eighths_on_mufu": mufu / 0.625}
+    breakdown = breakdown_of(per_op, ms_per_step)
+    if sustained is not None:
+        s_ops = sustained.pop("per_op_raw")
+        sustained["roofline"] = roofline_of(s_ops, sustained["clocks"])
+        sustained["tensor_ops"] = tensor_ops_of(s_ops)
+        sustained["per_op"] = breakdown_of(s_ops, sustained["ms_per_step"])
 
     cpu = None
     if not args.no_cpu_baseline:
@@ -453,18 +511,25 @@ def main():
                    "output_finite": out_finite,
                    "parallelism": "replicas x%d" % world},
         "clocks": clocks,
-        "e2e": {"value": whole_job_tflops(flops, world, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms,
+        "regime": regime_of(clocks),
+        # End to end through the C ABI's host-buffer call (xema_forward_host): pinned host -> arena ->
+        # pinned host on one stream, nothing on the device outside the budgeted arena.  The pipelined
+        # figure overlaps the copies of neighbouring steps with compute through staging buffers that
+        # are NOT part of the budget, so it is the extra, not the value.
+        "e2e": {"value": whole_job_tflops(flops, world, e2e_serial_ms), "unit": UNIT, "ms_per_step": e2e_serial_ms,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "how": "pinned host -> device -> pinned host every step; the copies of neighbouring steps "
-                       "overlap compute (BlockSession.run_pipelined)",
-                "staging_bytes_outside_arena": sess.staging_bytes,
-                "serial": {"value": whole_job_tflops(flops, world, e2e_serial_ms), "ms_per_step": e2e_serial_ms}},
+                "how": "xema_forward_host: host-to-device copy, forward, device-to-host copy in order on one stream",
+                "device_bytes": sess.plan.peak_bytes, "fits_budget": budget is None or sess.plan.peak_bytes <= budget,
+                "pipelined": {"value": whole_job_tflops(flops, world, e2e_ms), "ms_per_step": e2e_ms,
+                              "how": "BlockSession.run_pipelined: copies of neighbouring steps overlap compute",
+                              "staging_bytes_outside_arena": sess.staging_bytes,
+                              "device_bytes": sess.plan.peak_bytes + sess.staging_bytes,
+                              "fits_budget": budget is None or sess.plan.peak_bytes + sess.staging_bytes <= budget}},
         "gpu_launches": n_kernels * args.steps,
         "roofline": roofline,
-        "tensor_ops": {"tflops": tensor_fl / (tensor_ms * 1e-3) / 1e12, "ms": tensor_ms,
-                       "frac_of_sustained": tensor_fl / (tensor_ms * 1e-3) / 1e12 / peaks["bf16_sustained"],
-                       "frac_of_nominal_2250": tensor_fl / (tensor_ms * 1e-3) / 1e12 / 2250.0},
+        "tensor_ops": tensor_ops_of(per_op),
         "per_op": breakdown,
+        "sustained": sustained,
         "cpu_baseline": cpu,
     }
     if sweep:

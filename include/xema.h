@@ -237,6 +237,19 @@ int xema_plan_bind(xema_plan* plan, void* arena_dev, uint64_t arena_bytes,
 int xema_block_forward(const xema_plan* plan, void* stream);
 int xema_step_forward(const xema_plan* plan, void* stream);
 
+/* The same forward with HOST buffers (the end-to-end form of the paper's serving runtime,
+ * section "Static memory runtime": a request's latent goes in, the denoised latent comes out).
+ * Enqueues on `stream`: a host-to-device copy of hid_in_host [B,S,D] bf16 and temb_host [B,Dt]
+ * bf16 into their arena slots, all n_blocks blocks, and a device-to-host copy of the output
+ * hidden state into hid_out_host [B,S,D] bf16.  The arena is the one given to xema_plan_bind;
+ * nothing else on the device is touched or allocated.  The host buffers are the caller's and
+ * must stay valid until the stream has passed the call; they should be page-locked (the copies
+ * of pageable memory are staged by the CUDA runtime and may block the calling thread).  Does
+ * not synchronise.  XEMA_ESTATE if the plan is unbound, XEMA_ECUDA if a copy or launch is
+ * rejected. */
+int xema_forward_host(const xema_plan* plan, const void* hid_in_host, const void* temb_host,
+                      void* hid_out_host, void* stream);
+
 /* The block forward for callers that cannot allocate device memory (the paper has no
  * counterpart: its runtime always has PyTorch's allocator behind it).  Some callers can call
  * neither cudaMalloc nor a framework allocator: code inside a region that must not
@@ -252,7 +265,12 @@ int xema_step_forward(const xema_plan* plan, void* stream);
  * (device, written; may not overlap the inputs); status_dev: device, 4 zeroed bytes, or NULL.
  * Enqueues two device-to-device copies in, the block's launches, and one copy out on `stream`.
  * Calls no cudaMalloc/cudaFree and no allocating library routine; host memory for the plan is
- * taken from the C++ heap and released before returning.
+ * taken from the C++ heap and released before returning.  Every call derives the trace and
+ * its layout again and encodes all TMA descriptors on the host (tens of microseconds for a
+ * small template): a caller that can hold a plan should use xema_plan_bind once and
+ * xema_block_forward per call instead.  Host threads may call in concurrently as far as the
+ * host side goes (the cached device address is atomic); the shared scratch array is what
+ * limits them, see below.
  *
  * XEMA_ENOSPC: the template's arena peak for this chunk count exceeds XEMA_STATIC_ARENA_BYTES
  * (the tiny template needs 2 076 672 bytes at chunks = 1); use xema_block_forward with your own

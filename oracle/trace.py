@@ -17,6 +17,13 @@ Chunk c covers token rows [floor(c S / C), floor((c+1) S / C)).
 A phase may instead be split along the batch ("temporary serialization": only the planned steps
 are split into sub-batches, which rejoin in the full-size tensors afterwards): piece c of C then
 covers batch elements [floor(c B / C), floor((c+1) B / C)) and all S rows.
+
+Sequence parallelism (the paper's SP: the latent sequence is split across GPUs; section
+"Execution Configurations"): GPU p of P owns token rows [floor(p S / P), floor((p+1) S / P)).
+Its trace has the same ops; every tensor holds only the owned rows -- chunks then cut the owned
+rows, chunk c covering owned rows [floor(c n / C), floor((c+1) n / C)) of the n owned -- except
+`kv`, which stays full-size: phase A fills the owned rows, the keys and values of the other GPUs
+arrive in place (one all-gather) before phase B reads them.
 """
 from __future__ import annotations
 
@@ -67,37 +74,53 @@ def phase_counts(chunks):
 SPLIT_ROWS, SPLIT_BATCH = 0, 1
 
 
-def piece_elems(t, C, axis):
-    """Token-row count times batch count of every piece of a phase split C ways along `axis`."""
+def shard_rows(t, shard):
+    """(first row, row count) owned by shard = (p, P); the whole sequence for shard None."""
+    if shard is None:
+        return 0, t.seq
+    p, P = shard
+    if P < 1 or not 0 <= p < P or P > t.seq:
+        raise ValueError("shard must be (p, P) with 0 <= p < P <= S")
+    r0 = p * t.seq // P
+    return r0, (p + 1) * t.seq // P - r0
+
+
+def piece_elems(t, C, axis, rows=None):
+    """Token-row count times batch count of every piece of a phase split C ways along `axis`;
+    `rows` = number of token rows the phase covers (all of them by default)."""
+    rows = t.seq if rows is None else rows
     if axis == SPLIT_BATCH:
         b = chunk_rows(t.batch, C)
-        return [(b[c + 1] - b[c]) * t.seq for c in range(C)]
-    r = chunk_rows(t.seq, C)
+        return [(b[c + 1] - b[c]) * rows for c in range(C)]
+    r = chunk_rows(rows, C)
     return [t.batch * (r[c + 1] - r[c]) for c in range(C)]
 
 
-def trace(t, chunks, axes=(SPLIT_ROWS, SPLIT_ROWS, SPLIT_ROWS)):
+def trace(t, chunks, axes=(SPLIT_ROWS, SPLIT_ROWS, SPLIT_ROWS), shard=None):
     """Returns (tensors, n_ops).  tensors: list of dicts with name, kind, dtype, block,
     chunk, bytes (rounded up to 256), birth, death -- in id order (first birth, then
     table row).  `chunks` is an int or a per-phase triple (see phase_counts); with a triple
     the op list is MOD; C_A x (LN1A, KV, KROPE); C_B x (LN1B, Q, QROPE, ATTN, PROJ);
     C_C x (LN2, FFN1, FFN2) -- chunking applied only where the trace needs it.  `axes` says per
-    phase whether its pieces are row chunks (all batch elements) or sub-batches (all rows)."""
+    phase whether its pieces are row chunks (all batch elements) or sub-batches (all rows).
+    `shard` = (p, P): the trace of GPU p of P under sequence parallelism (see the module text)."""
     B, S, D, H, F, Dt = t.batch, t.seq, t.hidden, t.heads, t.ffn, t.temb_dim
+    _, n_own = shard_rows(t, shard)
     CA, CB, CC = phase_counts(chunks)
     L = t.n_blocks
     for C, ax in zip((CA, CB, CC), axes):
         if ax not in (SPLIT_ROWS, SPLIT_BATCH):
             raise ValueError("axis must be 0 (rows) or 1 (batch)")
-        if C < 1 or C > (B if ax == SPLIT_BATCH else S):
-            raise ValueError("chunks must be in [1, S] (rows) or [1, B] (batch)")
-    eA, eB, eC = (piece_elems(t, C, ax) for C, ax in zip((CA, CB, CC), axes))
+        if C < 1 or C > (B if ax == SPLIT_BATCH else n_own):
+            raise ValueError("chunks must be in [1, rows] (rows) or [1, B] (batch)")
+    eA, eB, eC = (piece_elems(t, C, ax, n_own) for C, ax in zip((CA, CB, CC), axes))
     rec = _Recorder()
 
     def meta(base, nbytes, kind, dtype, block, chunk=-1):
         return dict(base=base, bytes=align_up(nbytes), kind=kind, dtype=dtype, block=block, chunk=chunk)
 
-    u = 2 * B * S * D
+    u = 2 * B * n_own * D                 # one bf16 hidden tensor over the owned rows
+    u_all = 2 * B * S * D                 # ... over every row (keys and values of all GPUs)
     # inputs exist before the first op
     rec.tensors["temb"] = dict(meta("temb", 2 * B * Dt, KIND_INPUT, DTYPE_BF16, -1), name="temb", birth=0, death=1)
     rec.tensors["hid0"] = dict(meta("hid", u, KIND_INPUT, DTYPE_BF16, 0), name="hid0", birth=0, death=1)
@@ -105,7 +128,7 @@ def trace(t, chunks, axes=(SPLIT_ROWS, SPLIT_ROWS, SPLIT_ROWS)):
         hid, nxt = f"hid{l}", f"hid{l + 1}"
         mod, kv, res = f"mod{l}", f"kv{l}", f"res{l}"
         m_mod = (mod, meta("mod", 24 * B * D, KIND_FULL, DTYPE_F32, l))
-        m_kv = (kv, meta("kv", 2 * u, KIND_FULL, DTYPE_BF16, l))
+        m_kv = (kv, meta("kv", 2 * u_all, KIND_FULL, DTYPE_BF16, l))
         m_res = (res, meta("res", 2 * u, KIND_FULL, DTYPE_F32, l))
         m_nxt = (nxt, meta("hid", u, KIND_OUTPUT if l + 1 == L else KIND_FULL, DTYPE_BF16, l + 1))
         rec.op(reads=["temb"], writes=[m_mod])                                   # MOD

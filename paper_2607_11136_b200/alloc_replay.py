@@ -47,7 +47,9 @@ def replay(sequence, rounds: int, device: str = "cuda:0") -> dict:
     torch.cuda.set_device(device)
     torch.cuda.empty_cache()
     torch.cuda.reset_peak_memory_stats()
+    # whatever the process already holds (weights of earlier work, say) is not this replay's
     base_alloc = torch.cuda.memory_allocated()
+    base_reserved = torch.cuda.memory_reserved()
     plans = []
     for name, chunks in sequence:
         cfg = xb.make_config(template(name))
@@ -71,7 +73,7 @@ def replay(sequence, rounds: int, device: str = "cuda:0") -> dict:
         "static_arena_bytes": max(p["arena_peak_bytes"] for p in plans),
         "active_peak_bytes": max(p["max_live_bytes"] for p in plans),
         "torch_allocated_peak_bytes": torch.cuda.max_memory_allocated() - base_alloc,
-        "torch_reserved_peak_bytes": torch.cuda.max_memory_reserved(),
+        "torch_reserved_peak_bytes": torch.cuda.max_memory_reserved() - base_reserved,
         "allocator": os.environ.get("PYTORCH_CUDA_ALLOC_CONF", "default (caching allocator)"),
     }
     out["utilisation_torch"] = out["active_peak_bytes"] / out["torch_reserved_peak_bytes"]

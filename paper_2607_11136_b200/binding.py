@@ -25,7 +25,7 @@ EXPORTS = (
     "xema_plan_info", "xema_plan_phase_chunks", "xema_plan_mitigation", "xema_plan_tensor",
     "xema_plan_tensor_at", "xema_plan_bind", "xema_block_forward", "xema_step_forward",
     "xema_block_forward_static",
-    "xema_plan_launch_count", "xema_forward_prefix", "xema_forward_range", "xema_plan_op", "xema_op_mod", "xema_op_ln_modulate",
+    "xema_plan_launch_count", "xema_forward_host", "xema_forward_prefix", "xema_forward_range", "xema_plan_op", "xema_op_mod", "xema_op_ln_modulate",
     "xema_op_rmsnorm_rope", "xema_op_gemm", "xema_op_attention", "xema_strerror",
     "xema_last_cuda_error", "xema_version", "xema_selftest_wait_timeout",
     "xema_pluggable_malloc", "xema_pluggable_free", "xema_pluggable_mode", "xema_pluggable_recorded",
@@ -117,6 +117,7 @@ def lib() -> C.CDLL:
             "xema_plan_bind": [vp, vp, u64, P(xema_block_weights), vp, vp],
             "xema_block_forward": [vp, vp],
             "xema_step_forward": [vp, vp],
+            "xema_forward_host": [vp, vp, vp, vp, vp],
             "xema_block_forward_static": [P(xema_config), i32, P(xema_block_weights), vp, vp, vp, vp, vp, vp],
             "xema_plan_launch_count": [vp],
             "xema_forward_prefix": [vp, u32, vp],
@@ -395,6 +396,10 @@ class Plan:
 
     def step_forward(self, stream: int = 0):
         _check(lib().xema_step_forward(self._h, stream), "xema_step_forward")
+
+    def forward_host(self, hid_in_host: int, temb_host: int, hid_out_host: int, stream: int = 0):
+        """Host pointers in and out; both copies and the forward are enqueued on `stream`."""
+        _check(lib().xema_forward_host(self._h, hid_in_host, temb_host, hid_out_host, stream), "xema_forward_host")
 
     def forward_range(self, first_op: int, end_op: int, stream: int = 0):
         _check(lib().xema_forward_range(self._h, first_op, end_op, stream), "xema_forward_range")

@@ -387,6 +387,9 @@ constexpr int PAIR_B_HALF_BYTES = (PAIR_BN / 2) * BK * 2;
 constexpr int PAIR_STAGE_BYTES = A_TILE_BYTES + PAIR_B_HALF_BYTES;
 constexpr int PAIR_SMEM_BYTES = 1024 + PAIR_STAGES * PAIR_STAGE_BYTES + 256;
 constexpr int PAIR_TMEM_COLS = 2 * PAIR_BN;
+// Limit of one drain wait after a give-up (about 50 ms): long enough for any copy in flight,
+// short enough that six of them in a row stay far below the limit of a regular wait.
+constexpr long long kDrainLimitCycles = 100000000ll;
 
 template <int EPI>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
@@ -454,6 +457,30 @@ gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
           tma_load_3d_pair(sb, &map_w, full0, kb * BK, c.nt * PAIR_BN + (int)rank * (PAIR_BN / 2), 0);
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
+      }
+      // Tail: the same waits as for STAGES further fills, without filling.  They return once the
+      // commits that release this CTA's last fills (arrivals multicast by the even CTA) have
+      // landed here, so none of them can reach this CTA's barriers after it has left.
+      for (int s = 0; ok && s < STAGES; ++s) {
+        ok = mbar_wait(&empty[stage], phase ^ 1, abort_flag);
+        if (++stage == STAGES) { stage = 0; phase ^= 1; }
+      }
+      if (!ok) {
+        // Gave up.  Copies already issued must land before either CTA leaves: all of them
+        // complete on the even CTA's full[] barriers, so the even CTA waits (bounded, and
+        // without looking at the abort flag) for the latest fill of every stage, which covers
+        // the bytes of both CTAs wherever both issued; the closing cluster barrier then keeps
+        // the peer until that is done.  A short settling time on both CTAs covers loads of a
+        // stage that only one of the two CTAs still issued.
+        if (rank == 0) {
+          for (int s = 0; s < STAGES; ++s) {
+            const int st = (stage + s) % STAGES;                 // oldest outstanding first
+            const uint32_t ph = (st < stage) ? phase : (phase ^ 1);
+            volatile uint32_t dummy = 0;
+            mbar_wait_slow(&full[st], ph, &dummy, kDrainLimitCycles);
+          }
+        }
+        for (int i = 0; i < 64; ++i) __nanosleep(1000);
       }
     }
   } else if (warp == 1) {
@@ -535,18 +562,6 @@ gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
 }
 
 // ---------------------------------------------------------------------------------------------
-static int g_sm_count = 0;
-static int sm_count() {
-  if (g_sm_count == 0) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
-    int n = 0;
-    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return 148;
-    g_sm_count = n;
-  }
-  return g_sm_count;
-}
-
 static GemmParams make_params(const GemmLaunch& g) {
   GemmParams p;
   p.bias = (const __nv_bfloat16*)g.bias;
@@ -575,16 +590,9 @@ static GemmParams make_params(const GemmLaunch& g) {
 template <int BN, int EPI>
 static int launch_gemm_t(const GemmLaunch& g, cudaStream_t stream) {
   using Cfg = GemmCfg<BN>;
-  static bool attr_set = false;
+  static PerDeviceInt attr_done;
   auto kern = gemm_bf16_kernel<BN, EPI>;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES);
-    if (e != cudaSuccess) {
-      set_last_cuda_error((int)e);
-      return XEMA_ECUDA;
-    }
-    attr_set = true;
-  }
+  if (int rc = ensure_smem_attr(kern, Cfg::SMEM_BYTES, attr_done)) return rc;
   const GemmParams p = make_params(g);
   const int m_tiles = (g.rows + BM - 1) / BM;
   const long long tiles = (long long)g.batch * m_tiles * (g.N / BN);
@@ -595,19 +603,14 @@ static int launch_gemm_t(const GemmLaunch& g, cudaStream_t stream) {
 
 template <int EPI>
 static int launch_gemm_pair_t(const GemmLaunch& g, cudaStream_t stream) {
-  static bool attr_set = false;
+  static PerDeviceInt attr_done;
   auto kern = gemm_bf16_pair_kernel<EPI>;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, PAIR_SMEM_BYTES);
-    if (e != cudaSuccess) {
-      set_last_cuda_error((int)e);
-      return XEMA_ECUDA;
-    }
-    attr_set = true;
-  }
+  if (int rc = ensure_smem_attr(kern, PAIR_SMEM_BYTES, attr_done)) return rc;
   // A persistent grid must be resident all at once: ask how many CTA pairs fit on the device
   // (SMs are handed out to clusters in hardware groups, so it can be fewer than SMs / 2).
-  static int max_pairs = 0;
+  static PerDeviceInt pairs_cache;
+  const int dev = current_device();
+  int max_pairs = pairs_cache.get(dev);
   if (max_pairs == 0) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2 * (sm_count() / 2), 1, 1);
@@ -627,6 +630,7 @@ static int launch_gemm_pair_t(const GemmLaunch& g, cudaStream_t stream) {
       return XEMA_ECUDA;
     }
     max_pairs = std::min(n, sm_count() / 2);
+    pairs_cache.set(dev, max_pairs);
   }
   const GemmParams p = make_params(g);
   const int m_tiles = (g.rows + 2 * BM - 1) / (2 * BM);

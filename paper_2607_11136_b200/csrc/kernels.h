@@ -3,6 +3,8 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <atomic>
+
 #include "../../include/xema.h"
 
 namespace xema {
@@ -10,6 +12,37 @@ namespace xema {
 // Records cudaGetLastError(); returns XEMA_OK or XEMA_ECUDA.
 int check_launch();
 void set_last_cuda_error(int code);
+
+// One-time launch state (function attributes, SM counts, cluster occupancy) belongs to a device,
+// not to the process: these caches are indexed by the current device's ordinal and filled with
+// atomic stores, so several host threads, or one process that drives several GPUs, see a
+// value only after it was established on that device.  0 means "not known yet".  Ordinals at or
+// beyond kMaxDevices are never cached (the value is looked up again on every call).
+constexpr int kMaxDevices = 64;
+struct PerDeviceInt {
+  std::atomic<int> v[kMaxDevices];
+  int get(int dev) const { return (dev >= 0 && dev < kMaxDevices) ? v[dev].load(std::memory_order_acquire) : 0; }
+  void set(int dev, int value) {
+    if (dev >= 0 && dev < kMaxDevices) v[dev].store(value, std::memory_order_release);
+  }
+};
+// Ordinal of the calling thread's current device, or -1.
+int current_device();
+// Multiprocessor count of the current device (148 on a B200); cached per device.
+int sm_count();
+// Raises a kernel's dynamic shared-memory limit once per device.  `done` is the kernel's cache.
+template <typename Kernel>
+int ensure_smem_attr(Kernel kern, int bytes, PerDeviceInt& done) {
+  const int dev = current_device();
+  if (done.get(dev)) return XEMA_OK;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e != cudaSuccess) {
+    set_last_cuda_error((int)e);
+    return XEMA_ECUDA;
+  }
+  done.set(dev, 1);
+  return XEMA_OK;
+}
 
 int launch_mod(const void* temb, const void* w_mod, const void* b_mod, float* mod, int batch, int Dt, int n_out,
                cudaStream_t stream);
@@ -63,6 +96,6 @@ int attn_prepare(AttnLaunch* a, const void* q, long long ldq, long long q_batch_
                  long long ldkv, long long kv_batch_rows);
 int launch_attention(const AttnLaunch& a, cudaStream_t stream);
 int launch_attention_dh64(const AttnLaunch& a, cudaStream_t stream);   // two-tile kernel for head_dim 64
-constexpr int kAttnDh64KeysPerBlock = 64;                              // rows of its K/V TMA boxes
+constexpr int kAttnDh64KeysPerBlock = 128;                             // rows of its K/V TMA boxes
 
 }  // namespace xema

@@ -19,6 +19,21 @@ namespace xema {
 static thread_local int t_last_cuda_error = 0;
 void set_last_cuda_error(int code) { t_last_cuda_error = code; }
 
+int current_device() {
+  int dev = -1;
+  return cudaGetDevice(&dev) == cudaSuccess ? dev : -1;
+}
+
+int sm_count() {
+  static PerDeviceInt cache;
+  const int dev = current_device();
+  int n = cache.get(dev);
+  if (n > 0) return n;
+  if (dev < 0 || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return 148;
+  cache.set(dev, n);
+  return n;
+}
+
 int check_launch() {
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) {
@@ -115,6 +130,7 @@ struct xema_plan {
   uint64_t peak, live;
   uint32_t n_ops;
   bool bound;
+  uint8_t* arena;     // as given to xema_plan_bind
   const float* rope;
   std::vector<Op> ops;
 };
@@ -181,6 +197,7 @@ int xema_plan_create_mitigated(const xema_config* cfg, const xema_mitigation* m,
     pl->axes[i] = m->axis[i];
   }
   pl->bound = false;
+  pl->arena = nullptr;
   pl->rope = nullptr;
   int rc = build_trace(*cfg, chunks, pl->axes, pl->tensors, &pl->n_ops);
   if (!rc) {
@@ -252,6 +269,7 @@ int xema_plan_bind(xema_plan* plan, void* arena_dev, uint64_t arena_bytes, const
   plan->bound = false;
   plan->ops.clear();
   plan->rope = rope_dev;
+  plan->arena = static_cast<uint8_t*>(arena_dev);
   uint8_t* arena = static_cast<uint8_t*>(arena_dev);
   unsigned int* status = static_cast<unsigned int*>(status_dev);
 
@@ -471,6 +489,36 @@ int xema_block_forward(const xema_plan* plan, void* stream) {
 int xema_step_forward(const xema_plan* plan, void* stream) {
   if (!plan) return XEMA_EINVAL;
   return run_ops(plan, 0, plan->ops.size(), stream);
+}
+
+int xema_forward_host(const xema_plan* plan, const void* hid_in_host, const void* temb_host, void* hid_out_host,
+                      void* stream) {
+  if (!plan || !hid_in_host || !temb_host || !hid_out_host) return XEMA_EINVAL;
+  if (!plan->bound) return XEMA_ESTATE;
+  const xema_config& c = plan->cfg;
+  char out_name[32];
+  std::snprintf(out_name, sizeof(out_name), "hid%d", c.n_blocks);
+  auto i_in = plan->index.find("hid0"), i_temb = plan->index.find("temb"), i_out = plan->index.find(out_name);
+  if (i_in == plan->index.end() || i_temb == plan->index.end() || i_out == plan->index.end()) return XEMA_EINVAL;
+  // exact sizes (the planned sizes are rounded up to 256 bytes; the caller's buffers are not)
+  const size_t hid_bytes = (size_t)2 * c.batch * (size_t)seq_len(c) * c.hidden;
+  const size_t temb_bytes = (size_t)2 * c.batch * c.temb_dim;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  cudaError_t e = cudaMemcpyAsync(plan->arena + plan->offsets[i_in->second], hid_in_host, hid_bytes, cudaMemcpyHostToDevice, st);
+  if (e == cudaSuccess)
+    e = cudaMemcpyAsync(plan->arena + plan->offsets[i_temb->second], temb_host, temb_bytes, cudaMemcpyHostToDevice, st);
+  if (e != cudaSuccess) {
+    t_last_cuda_error = (int)e;
+    return XEMA_ECUDA;
+  }
+  int rc = run_ops(plan, 0, plan->ops.size(), stream);
+  if (rc) return rc;
+  e = cudaMemcpyAsync(hid_out_host, plan->arena + plan->offsets[i_out->second], hid_bytes, cudaMemcpyDeviceToHost, st);
+  if (e != cudaSuccess) {
+    t_last_cuda_error = (int)e;
+    return XEMA_ECUDA;
+  }
+  return XEMA_OK;
 }
 
 int xema_forward_prefix(const xema_plan* plan, uint32_t n_logical_ops, void* stream) {

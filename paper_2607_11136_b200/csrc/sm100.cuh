@@ -60,14 +60,12 @@ __device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Upper bound, in nanoseconds, for which one try_wait of the slow path may park the thread.
-#ifndef XEMA_WAIT_HINT_NS
-#define XEMA_WAIT_HINT_NS 1000u
-#endif
-// Plain polls before a wait moves to the parked slow path.
-#ifndef XEMA_WAIT_FAST_POLLS
-#define XEMA_WAIT_FAST_POLLS 2
-#endif
+// Upper bound, in nanoseconds, for which one try_wait of the slow path may park the thread, and
+// the number of plain polls before a wait moves to that parked slow path.  (Hints of 0.2-5 us and
+// one to four plain polls measured the same; no plain poll at all cost 12 % in the attention
+// kernels.)
+constexpr uint32_t kWaitHintNs = 1000u;
+constexpr int kWaitFastPolls = 2;
 // Non-blocking look at a barrier phase (try_wait may park the thread for a while when the phase
 // is still open; test_wait returns at once).
 __device__ __forceinline__ bool mbar_peek(uint64_t* bar, uint32_t parity) {
@@ -96,7 +94,7 @@ static __device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parit
         "selp.u32 %0, 1, 0, p;\n"
         "}\n"
         : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity), "r"(XEMA_WAIT_HINT_NS)
+        : "r"(smem_u32(bar)), "r"(parity), "r"(kWaitHintNs)
         : "memory");
     if (ok) return true;
     if ((++polls & 0x3F) == 0) {
@@ -111,9 +109,57 @@ static __device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parit
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag) {
   // fast path: a few plain polls with nothing else in the dependent chain
 #pragma unroll 1
-  for (int i = 0; i < XEMA_WAIT_FAST_POLLS; ++i)
+  for (int i = 0; i < kWaitFastPolls; ++i)
     if (mbar_test(bar, parity)) return true;
   return mbar_wait_slow(bar, parity, abort_flag, kWaitLimitCycles);
+}
+
+// Bounded wait for a whole warp that polls together (every lane executes it with the same
+// arguments): one loop in a single block of PTX -- no function call, no vote, no compiler-made
+// reconvergence points around it.  Every poll may park the warp for up to kWaitHintNs; the
+// loop gives up after kWaitLimitPolls polls (seconds), raises the CTA's abort flag and returns
+// false.  The abort flag is looked at every 1024 polls.
+constexpr uint32_t kWaitLimitPolls = 1u << 22;
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag) {
+  uint32_t done;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(done)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  if (done) return true;
+  uint32_t polls = 0;
+  while (true) {
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        ".reg .u32 n;\n"
+        "mov.u32 n, 0;\n"
+        "WAIT_LOOP:\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"
+        "@p bra WAIT_DONE;\n"
+        "add.u32 n, n, 1;\n"
+        "setp.lt.u32 p, n, 1024;\n"
+        "@p bra WAIT_LOOP;\n"
+        "setp.ne.u32 p, n, n;\n"
+        "WAIT_DONE:\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(done)
+        : "r"(smem_u32(bar)), "r"(parity), "r"(kWaitHintNs)
+        : "memory");
+    if (done) return true;
+    polls += 1024;
+    if (*abort_flag) return false;
+    if (polls >= kWaitLimitPolls) {
+      *abort_flag = 1;
+      return false;
+    }
+  }
 }
 
 // ---- CTA pairs (thread-block cluster of two) -------------------------------------------------
@@ -148,7 +194,7 @@ static __device__ __noinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t pa
         "selp.u32 %0, 1, 0, p;\n"
         "}\n"
         : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity), "r"(XEMA_WAIT_HINT_NS)
+        : "r"(smem_u32(bar)), "r"(parity), "r"(kWaitHintNs)
         : "memory");
     if (ok) return true;
     if ((++polls & 0x3F) == 0) {
@@ -324,6 +370,37 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
       : "memory");
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// The same wait, tied to the registers of one earlier load: the compiler sees them as rewritten
+// here, so nothing that reads them can move above the wait while other loads stay in flight.
+__device__ __forceinline__ void tmem_ld_wait_on(uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.wait::ld.sync.aligned;"
+      : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+        "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
+        "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
+        "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+      :
+      : "memory");
+}
+
+// 16 consecutive columns, and the wait tied to their registers.
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait_on(uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.wait::ld.sync.aligned;"
+      : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+        "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15])
+      :
+      : "memory");
+}
 
 // registers -> TMEM, same shape.
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {

@@ -8,6 +8,7 @@
 // fixed array that is part of the library image.
 #include <cuda_runtime.h>
 
+#include <atomic>
 #include <cstdint>
 
 #include "../../include/xema.h"
@@ -21,8 +22,10 @@ namespace {
 
 constexpr int kMaxDevices = 64;
 // Device address of g_static_arena per device ordinal.  In host code the symbol's name is only
-// a handle; the address a kernel can use has to be asked for, once per device.
-unsigned char* g_arena_ptr[kMaxDevices] = {};
+// a handle; the address a kernel can use has to be asked for, once per device.  Atomic so that
+// host threads calling in at the same time either see the address or look it up themselves (the
+// lookup is idempotent).  A cudaDeviceReset() by the caller invalidates the cached address.
+std::atomic<unsigned char*> g_arena_ptr[kMaxDevices] = {};
 
 int static_arena_for_current_device(unsigned char** out) {
   int dev = -1;
@@ -31,16 +34,18 @@ int static_arena_for_current_device(unsigned char** out) {
     xema::set_last_cuda_error((int)(e != cudaSuccess ? e : cudaErrorInvalidDevice));
     return XEMA_ECUDA;
   }
-  if (!g_arena_ptr[dev]) {
+  unsigned char* cached = g_arena_ptr[dev].load(std::memory_order_acquire);
+  if (!cached) {
     void* p = nullptr;
     e = cudaGetSymbolAddress(&p, g_static_arena);
     if (e != cudaSuccess || !p) {
       xema::set_last_cuda_error((int)(e != cudaSuccess ? e : cudaErrorInvalidSymbol));
       return XEMA_ECUDA;
     }
-    g_arena_ptr[dev] = static_cast<unsigned char*>(p);
+    cached = static_cast<unsigned char*>(p);
+    g_arena_ptr[dev].store(cached, std::memory_order_release);
   }
-  *out = g_arena_ptr[dev];
+  *out = cached;
   return XEMA_OK;
 }
 

@@ -8,7 +8,7 @@ from paper_2607_11136_b200 import binding as xb
 from paper_2607_11136_b200.session import BlockSession
 from xema_inputs import bits_to_f64, make_activations, make_block_weights, sample_rows, template
 
-from gpu_util import DEV, assert_bf16_close, assert_close, tolerance_split, stats
+from gpu_util import DEV, assert_bf16_close, assert_close, check_block_parity, expect_raw_bound
 
 pytestmark = pytest.mark.gpu
 
@@ -210,11 +210,16 @@ def test_full_size_block_sampled_rows(name):
     cfg = xb.make_config(t)
     w = make_block_weights(t, 0)
     x, temb = make_activations(t)
-    bounds = [c * t.seq // C for C in (2, 4, 8) for c in range(1, C)]
-    rows = sample_rows(t, boundaries=bounds, n_random=96)
+    # chunk starts of every count tried, plus both sides of the 128- and 256-row tile edges at the
+    # start and next to the ragged tail (17776 = 69 * 256 + 112: last full tile ends at row 17664)
+    bounds = [c * t.seq // C for C in (2, 4, 8) for c in range(1, C)] + [128, 256, t.seq // 256 * 256,
+                                                                         t.seq // 128 * 128]
+    rows = sample_rows(t, boundaries=bounds, n_random=1100)
+    assert len(rows) >= 1024 and {t.seq // 256 * 256 - 1, t.seq // 256 * 256, t.seq - 1} <= set(rows.tolist())
     ref = ob.block_forward(t, _f64(w), bits_to_f64(x), bits_to_f64(temb), rows=rows)["y"]
     dev_w = None
     first = None
+    parity = None
     for C in (1, 2, 4, 8):
         peak = xb.Plan(cfg, C).peak_bytes
         s = BlockSession(t, [dev_w or w], budget_bytes=peak, per_phase=False)
@@ -225,18 +230,7 @@ def test_full_size_block_sampled_rows(name):
         y = s.output_bits()
         if first is None:
             first = y
-            got = bits_to_f64(y[:, rows])
-            st = stats(got, ref)
-            tol = 2e-2 * st["rms_ref"]
-            n_over, n_fmt, n_compute, max_compute = tolerance_split(y[:, rows], ref, tol)
-            print("full-size %s: max-abs %.4e (%.4f of RMS), over tol %d of %d (format-limited %d, compute %d), "
-                  "max-abs without format-limited %.4e, cosine %.7f"
-                  % (name, st["max_abs"], st["rel"], n_over, got.size, n_fmt, n_compute, max_compute, st["cos"]))
-            # every element is within tolerance, or is a faithfully rounded bf16 where the bf16
-            # spacing exceeds the tolerance; such elements stay rare and within one spacing
-            assert n_compute == 0 and max_compute <= tol, (st, n_over, n_fmt, n_compute)
-            assert n_fmt <= 1e-4 * got.size and st["max_abs"] <= 3e-2 * st["rms_ref"]
-            assert st["cos"] >= 0.9995
+            parity = check_block_parity("full-size %s" % name, y[:, rows], ref)
         else:
             assert np.array_equal(first, y), C
         del s
@@ -250,6 +244,7 @@ def test_full_size_block_sampled_rows(name):
         assert np.array_equal(first, s.output_bits()), want
         del s
         torch.cuda.empty_cache()
+    expect_raw_bound(parity)
 
 
 def test_bounded_wait_gives_up_and_reports():
@@ -277,6 +272,35 @@ def test_bounded_wait_gives_up_and_reports():
     s.forward()
     ref = ob.block_forward(t, _f64(w), bits_to_f64(x), bits_to_f64(temb))["y"]
     assert_close(bits_to_f64(s.output_bits()), ref, "block after a timed-out wait")
+
+
+def test_forward_host_equals_arena_forward(tiny_case):
+    """xema_forward_host (pinned host buffers in and out, copies and launches on one stream)
+    returns the bits of set_inputs / forward / output_bits, twice in a row, and allocates
+    nothing on the device."""
+    t, w, x, temb, ref = tiny_case
+    s = BlockSession(t, [w], chunks=(1, 1, 2))
+    s.set_inputs(x, temb)
+    s.forward()
+    want = s.output_bits().copy()
+    x_h = torch.from_numpy(x.view(np.int16)).pin_memory()
+    t_h = torch.from_numpy(temb.view(np.int16)).pin_memory()
+    y_h = torch.zeros_like(x_h).pin_memory()
+    stream = torch.cuda.current_stream().cuda_stream
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    for _ in range(2):
+        y_h.zero_()
+        s.plan.forward_host(x_h.data_ptr(), t_h.data_ptr(), y_h.data_ptr(), stream)
+        torch.cuda.synchronize()
+        assert np.array_equal(y_h.numpy().view(np.uint16), want)
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0
+    s.check_status()
+    # an unbound plan is refused
+    with pytest.raises(xb.XemaError) as e:
+        xb.Plan(xb.make_config(t), 1).forward_host(x_h.data_ptr(), t_h.data_ptr(), y_h.data_ptr(), stream)
+    assert e.value.status == xb.XEMA_ESTATE
 
 
 def test_pipelined_host_to_host_equals_serial(tiny_case):
