@@ -188,6 +188,24 @@ int xema_trace_mitigated(const xema_config* cfg, const xema_mitigation* m, xema_
 int xema_mitigation_for_budget(const xema_config* cfg, uint64_t budget_bytes, int32_t max_chunks,
                                xema_mitigation* m, uint64_t* peak_bytes);
 
+/* ---- sequence parallelism (the paper's SP, section "Execution Configurations": the latent
+ * sequence is split across GPUs; the planner enumerates the SP degree in stage 1 of "Planning
+ * Workflow") ---------------------------------------------------------------------------------
+ * GPU `shard` of `shards` owns token rows [floor(shard*S/shards), floor((shard+1)*S/shards)).
+ * Its block has the same ops.  Every tensor holds the owned rows only (chunks then cut the owned
+ * rows: chunk c of C covers owned rows [floor(c*n/C), floor((c+1)*n/C)) of the n owned), except
+ * kv<l>, which stays [B, S, 2D] over ALL rows: phase A (LN1A, KV, KROPE) fills the owned rows,
+ * the keys and values of the other GPUs must be in place (one all-gather, done by the caller
+ * into its own arena) before the first op of phase B.  Nothing in the library communicates. */
+
+/* First row and number of rows shard `shard` of `shards` owns.  XEMA_EINVAL unless
+ * 0 <= shard < shards <= S. */
+int xema_shard_rows(const xema_config* cfg, int32_t shard, int32_t shards, int64_t* row0, int64_t* rows);
+/* xema_trace_mitigated for one shard (shard 0 of 1 gives the same trace).  Counts are limited by
+ * the owned rows. */
+int xema_trace_sharded(const xema_config* cfg, const xema_mitigation* m, int32_t shard, int32_t shards,
+                       xema_tensor* out, size_t cap, size_t* n_tensors, uint32_t* n_ops);
+
 /* RoPE table for the template: host_out (host) receives S * (dh/2) * 2 floats laid out
  * [token][pair][cos, sin]; angle = position * rope_base^(-2j/d) inside each of the three
  * sections (t, h, w), evaluated in double precision and rounded once.  Text tokens sit at
@@ -213,6 +231,20 @@ int xema_plan_phase_chunks(const xema_plan* plan, int32_t chunks[3]);
 /* Plan with a split axis per phase (see xema_trace_mitigated), and the plan's counts and axes. */
 int xema_plan_create_mitigated(const xema_config* cfg, const xema_mitigation* m, xema_plan** out);
 int xema_plan_mitigation(const xema_plan* plan, xema_mitigation* m);
+/* Plan for one sequence-parallel shard (see xema_trace_sharded).  Its hid<l> / res<l> tensors and
+ * its input and output are [B, rows owned, D]; token positions (RoPE) stay global.  The forward
+ * calls run as usual; the caller splits them at the gather points:
+ *   for every block l: xema_forward_range(plan, previous point, first_op(l)); all-gather of
+ *   kv<l>'s rows; ... and xema_forward_range(plan, first_op(last), n_ops) at the end.
+ * xema_forward_host refuses a sharded plan (XEMA_ESTATE). */
+int xema_plan_create_sharded(const xema_config* cfg, const xema_mitigation* m, int32_t shard, int32_t shards,
+                             xema_plan** out);
+/* The plan's shard and the rows it owns (0 of 1 and all rows for an unsharded plan). */
+int xema_plan_shard(const xema_plan* plan, int32_t* shard, int32_t* shards, int64_t* row0, int64_t* rows);
+/* Gather point of block `block`: *first_op = index of the first op of its phase B (every op
+ * before it may run before the exchange, none from it on); *kv_offset = arena offset of kv<block>,
+ * laid out [B, S, 2D] bf16 with row (b, r) at ((b*S + r) * 2D) elements, K half first. */
+int xema_plan_gather_point(const xema_plan* plan, int32_t block, uint32_t* first_op, uint64_t* kv_offset);
 /* Offset and (256-rounded) size of a tensor by name, e.g. "hid0", "temb", "hid1", "res0". */
 int xema_plan_tensor(const xema_plan* plan, const char* name, uint64_t* offset, uint64_t* bytes);
 /* Copy of the plan's tensor i and its offset. */

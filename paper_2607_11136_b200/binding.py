@@ -25,6 +25,7 @@ EXPORTS = (
     "xema_plan_info", "xema_plan_phase_chunks", "xema_plan_mitigation", "xema_plan_tensor",
     "xema_plan_tensor_at", "xema_plan_bind", "xema_block_forward", "xema_step_forward",
     "xema_block_forward_static",
+    "xema_shard_rows", "xema_trace_sharded", "xema_plan_create_sharded", "xema_plan_shard", "xema_plan_gather_point",
     "xema_plan_launch_count", "xema_forward_host", "xema_forward_prefix", "xema_forward_range", "xema_plan_op", "xema_op_mod", "xema_op_ln_modulate",
     "xema_op_rmsnorm_rope", "xema_op_gemm", "xema_op_attention", "xema_strerror",
     "xema_last_cuda_error", "xema_version", "xema_selftest_wait_timeout",
@@ -99,6 +100,11 @@ def lib() -> C.CDLL:
             "xema_trace_mitigated": [P(xema_config), P(xema_mitigation), P(xema_tensor), sz, P(sz), P(u32)],
             "xema_mitigation_for_budget": [P(xema_config), u64, i32, P(xema_mitigation), P(u64)],
             "xema_plan_create_mitigated": [P(xema_config), P(xema_mitigation), P(vp)],
+            "xema_plan_create_sharded": [P(xema_config), P(xema_mitigation), i32, i32, P(vp)],
+            "xema_trace_sharded": [P(xema_config), P(xema_mitigation), i32, i32, P(xema_tensor), sz, P(sz), P(u32)],
+            "xema_shard_rows": [P(xema_config), i32, i32, P(i64), P(i64)],
+            "xema_plan_shard": [vp, P(i32), P(i32), P(i64), P(i64)],
+            "xema_plan_gather_point": [vp, i32, P(u32), P(u64)],
             "xema_plan_mitigation": [vp, P(xema_mitigation)],
             "xema_plan_phase_chunks": [vp, P(i32)],
             "xema_plan_arena": [P(xema_tensor), sz, P(u64), P(u64), P(u64)],
@@ -233,6 +239,27 @@ def xema_trace_mitigated(cfg: xema_config, chunks, axes):
     return [_tensor_dict(t) for t in arr], ops.value
 
 
+def xema_trace_sharded(cfg: xema_config, chunks, axes, shard: int, shards: int):
+    """The trace of sequence-parallel shard `shard` of `shards` -> (tensor dicts, n_ops)"""
+    c3 = (chunks,) * 3 if isinstance(chunks, int) else chunks
+    m = _mitigation(c3, axes or (SPLIT_ROWS,) * 3)
+    n, ops = C.c_size_t(0), C.c_uint32(0)
+    rc = lib().xema_trace_sharded(C.byref(cfg), C.byref(m), shard, shards, None, 0, C.byref(n), C.byref(ops))
+    if rc != XEMA_ENOSPC:
+        _check(rc, "xema_trace_sharded")
+    arr = (xema_tensor * n.value)()
+    _check(lib().xema_trace_sharded(C.byref(cfg), C.byref(m), shard, shards, arr, n.value, C.byref(n), C.byref(ops)),
+           "xema_trace_sharded")
+    return [_tensor_dict(t) for t in arr], ops.value
+
+
+def xema_shard_rows(cfg: xema_config, shard: int, shards: int):
+    """-> (first row, rows) owned by the shard"""
+    r0, n = C.c_int64(0), C.c_int64(0)
+    _check(lib().xema_shard_rows(C.byref(cfg), shard, shards, C.byref(r0), C.byref(n)), "xema_shard_rows")
+    return r0.value, n.value
+
+
 def xema_mitigation_for_budget(cfg: xema_config, budget_bytes: int, max_chunks: int):
     """-> ((C_A, C_B, C_C), axes, peak_bytes); counts and axes are None when nothing fits."""
     m, peak = xema_mitigation(), C.c_uint64(0)
@@ -325,12 +352,18 @@ def xema_rope_table(cfg: xema_config) -> np.ndarray:
 class Plan:
     """Owner of an xema_plan handle."""
 
-    def __init__(self, cfg: xema_config, chunks, axes=None):
+    def __init__(self, cfg: xema_config, chunks, axes=None, shard=None):
         """chunks: one count (xema_plan_create) or a per-phase triple (xema_plan_create_phases);
-        with `axes` (per-phase SPLIT_ROWS / SPLIT_BATCH) xema_plan_create_mitigated."""
+        with `axes` (per-phase SPLIT_ROWS / SPLIT_BATCH) xema_plan_create_mitigated; with
+        `shard` = (p, P) xema_plan_create_sharded (the plan of one sequence-parallel shard)."""
         self.cfg = cfg
         self._h = C.c_void_p()
-        if axes is not None:
+        if shard is not None:
+            c3 = (chunks,) * 3 if isinstance(chunks, int) else chunks
+            m = _mitigation(c3, axes or (SPLIT_ROWS,) * 3)
+            _check(lib().xema_plan_create_sharded(C.byref(cfg), C.byref(m), shard[0], shard[1], C.byref(self._h)),
+                   "xema_plan_create_sharded")
+        elif axes is not None:
             c3 = (chunks,) * 3 if isinstance(chunks, int) else chunks
             _check(lib().xema_plan_create_mitigated(C.byref(cfg), C.byref(_mitigation(c3, axes)), C.byref(self._h)),
                    "xema_plan_create_mitigated")
@@ -350,7 +383,17 @@ class Plan:
         m = xema_mitigation()
         _check(lib().xema_plan_mitigation(self._h, C.byref(m)), "xema_plan_mitigation")
         self.axes = tuple(m.axis)
+        p_, P_, r0, n = C.c_int32(), C.c_int32(), C.c_int64(), C.c_int64()
+        _check(lib().xema_plan_shard(self._h, C.byref(p_), C.byref(P_), C.byref(r0), C.byref(n)), "xema_plan_shard")
+        self.shard, self.row0, self.rows = (p_.value, P_.value), r0.value, n.value
         self._keep = None
+
+    def gather_point(self, block: int):
+        """-> (index of the first op that needs every shard's keys and values of `block`,
+        arena offset of its kv tensor [B, S, 2D])"""
+        op, off = C.c_uint32(), C.c_uint64()
+        _check(lib().xema_plan_gather_point(self._h, block, C.byref(op), C.byref(off)), "xema_plan_gather_point")
+        return op.value, off.value
 
     def close(self):
         if self._h:

@@ -79,9 +79,26 @@ int build_trace(const xema_config& cfg, const int32_t chunks[3], std::vector<xem
 
 int build_trace(const xema_config& cfg, const int32_t chunks[3], const int32_t axes[3], std::vector<xema_tensor>& out,
                 uint32_t* n_ops) {
+  return build_trace(cfg, chunks, axes, Shard{}, out, n_ops);
+}
+
+int shard_rows(const xema_config& cfg, Shard sh, int64_t* row0, int64_t* rows) {
+  const int64_t S = seq_len(cfg);
+  if (sh.P < 1 || sh.p < 0 || sh.p >= sh.P || sh.P > S) return XEMA_EINVAL;
+  const int64_t r0 = (int64_t)sh.p * S / sh.P;
+  if (row0) *row0 = r0;
+  if (rows) *rows = (int64_t)(sh.p + 1) * S / sh.P - r0;
+  return XEMA_OK;
+}
+
+int build_trace(const xema_config& cfg, const int32_t chunks[3], const int32_t axes[3], Shard sh,
+                std::vector<xema_tensor>& out, uint32_t* n_ops) {
   int rc = validate_config(cfg);
   if (rc) return rc;
-  const int64_t S = seq_len(cfg);
+  const int64_t S_all = seq_len(cfg);
+  int64_t S = 0;                       // rows this trace covers: the owned rows of the shard
+  rc = shard_rows(cfg, sh, nullptr, &S);
+  if (rc) return rc;
   for (int i = 0; i < 3; ++i) {
     if (axes[i] != XEMA_SPLIT_ROWS && axes[i] != XEMA_SPLIT_BATCH) return XEMA_EINVAL;
     if (chunks[i] < 1 || chunks[i] > (axes[i] == XEMA_SPLIT_BATCH ? (int64_t)cfg.batch : S)) return XEMA_EINVAL;
@@ -91,7 +108,8 @@ int build_trace(const xema_config& cfg, const int32_t chunks[3], const int32_t a
   const uint32_t L = (uint32_t)cfg.n_blocks;
   const uint32_t ops_per_block = 1 + 3 * CA + 5 * CB + 3 * CC;
   const uint32_t total_ops = L * ops_per_block;
-  const uint64_t u = 2 * B * (uint64_t)S * D;
+  const uint64_t u = 2 * B * (uint64_t)S * D;           // one bf16 hidden tensor over the owned rows
+  const uint64_t u_all = 2 * B * (uint64_t)S_all * D;   // ... over every row: keys and values of all shards
   // rows x batch elements of piece c of a phase split C ways along its axis
   auto elems_of = [&](uint32_t c, uint32_t C, int phase) {
     if (axes[phase] == XEMA_SPLIT_BATCH)
@@ -117,7 +135,7 @@ int build_trace(const xema_config& cfg, const int32_t chunks[3], const int32_t a
       uint64_t n = elems_of(c, CA, 0);
       out.push_back(make("h1a", l, c, XEMA_KIND_CHUNK, XEMA_DTYPE_BF16, 2 * n * D, op.ln1a(c), op.kv(c) + 1));
       if (c == 0)
-        out.push_back(make("kv", l, -1, XEMA_KIND_FULL, XEMA_DTYPE_BF16, 2 * u, op.kv(0), op.attn(CB - 1) + 1));
+        out.push_back(make("kv", l, -1, XEMA_KIND_FULL, XEMA_DTYPE_BF16, 2 * u_all, op.kv(0), op.attn(CB - 1) + 1));
     }
     for (uint32_t c = 0; c < CB; ++c) {
       uint64_t n = elems_of(c, CB, 1);
@@ -402,6 +420,33 @@ int xema_trace_mitigated(const xema_config* cfg, const xema_mitigation* m, xema_
   if (cap < ts.size() || !out) return XEMA_ENOSPC;
   std::memcpy(out, ts.data(), ts.size() * sizeof(xema_tensor));
   return XEMA_OK;
+}
+
+int xema_trace_sharded(const xema_config* cfg, const xema_mitigation* m, int32_t shard, int32_t shards,
+                       xema_tensor* out, size_t cap, size_t* n_tensors, uint32_t* n_ops) {
+  if (!cfg || !m) return XEMA_EINVAL;
+  std::vector<xema_tensor> ts;
+  uint32_t ops = 0;
+  xema::Shard sh;
+  sh.p = shard;
+  sh.P = shards;
+  int rc = xema::build_trace(*cfg, m->chunks, m->axis, sh, ts, &ops);
+  if (rc) return rc;
+  if (n_tensors) *n_tensors = ts.size();
+  if (n_ops) *n_ops = ops;
+  if (cap < ts.size() || !out) return XEMA_ENOSPC;
+  std::memcpy(out, ts.data(), ts.size() * sizeof(xema_tensor));
+  return XEMA_OK;
+}
+
+int xema_shard_rows(const xema_config* cfg, int32_t shard, int32_t shards, int64_t* row0, int64_t* rows) {
+  if (!cfg) return XEMA_EINVAL;
+  int rc = xema::validate_config(*cfg);
+  if (rc) return rc;
+  xema::Shard sh;
+  sh.p = shard;
+  sh.P = shards;
+  return xema::shard_rows(*cfg, sh, row0, rows);
 }
 
 int xema_mitigation_for_budget(const xema_config* cfg, uint64_t budget_bytes, int32_t max_chunks,

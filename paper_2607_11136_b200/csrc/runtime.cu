@@ -124,6 +124,7 @@ struct xema_plan {
   xema_config cfg;
   int32_t chunks[3];  // key/value, attention, feed-forward phase
   int32_t axes[3];    // XEMA_SPLIT_ROWS or XEMA_SPLIT_BATCH per phase
+  Shard shard;        // sequence-parallel shard this plan covers ({0, 1}: the whole sequence)
   std::vector<xema_tensor> tensors;
   std::vector<uint64_t> offsets;
   std::unordered_map<std::string, size_t> index;
@@ -186,6 +187,11 @@ int xema_plan_create_phases(const xema_config* cfg, const int32_t chunks[3], xem
 }
 
 int xema_plan_create_mitigated(const xema_config* cfg, const xema_mitigation* m, xema_plan** out) {
+  return xema_plan_create_sharded(cfg, m, 0, 1, out);
+}
+
+int xema_plan_create_sharded(const xema_config* cfg, const xema_mitigation* m, int32_t shard, int32_t shards,
+                             xema_plan** out) {
   if (!cfg || !out || !m) return XEMA_EINVAL;
   *out = nullptr;
   xema_plan* pl = new (std::nothrow) xema_plan();
@@ -199,7 +205,9 @@ int xema_plan_create_mitigated(const xema_config* cfg, const xema_mitigation* m,
   pl->bound = false;
   pl->arena = nullptr;
   pl->rope = nullptr;
-  int rc = build_trace(*cfg, chunks, pl->axes, pl->tensors, &pl->n_ops);
+  pl->shard.p = shard;
+  pl->shard.P = shards;
+  int rc = build_trace(*cfg, chunks, pl->axes, pl->shard, pl->tensors, &pl->n_ops);
   if (!rc) {
     pl->offsets.assign(pl->tensors.size(), 0);
     rc = plan_arena(pl->tensors.data(), pl->tensors.size(), pl->offsets.data(), &pl->peak, &pl->live);
@@ -237,6 +245,25 @@ int xema_plan_mitigation(const xema_plan* plan, xema_mitigation* m) {
   for (int i = 0; i < 3; ++i) {
     m->chunks[i] = plan->chunks[i];
     m->axis[i] = plan->axes[i];
+  }
+  return XEMA_OK;
+}
+
+int xema_plan_shard(const xema_plan* plan, int32_t* shard, int32_t* shards, int64_t* row0, int64_t* rows) {
+  if (!plan) return XEMA_EINVAL;
+  if (shard) *shard = plan->shard.p;
+  if (shards) *shards = plan->shard.P;
+  return shard_rows(plan->cfg, plan->shard, row0, rows);
+}
+
+int xema_plan_gather_point(const xema_plan* plan, int32_t block, uint32_t* first_op, uint64_t* kv_offset) {
+  if (!plan || block < 0 || block >= plan->cfg.n_blocks) return XEMA_EINVAL;
+  const uint32_t per_block = 1 + 3 * (uint32_t)plan->chunks[0] + 5 * (uint32_t)plan->chunks[1] + 3 * (uint32_t)plan->chunks[2];
+  if (first_op) *first_op = (uint32_t)block * per_block + 1 + 3 * (uint32_t)plan->chunks[0];
+  if (kv_offset) {
+    auto it = plan->index.find("kv" + std::to_string(block));
+    if (it == plan->index.end()) return XEMA_EINVAL;
+    *kv_offset = plan->offsets[it->second];
   }
   return XEMA_OK;
 }
@@ -288,7 +315,12 @@ int xema_plan_bind(xema_plan* plan, void* arena_dev, uint64_t arena_bytes, const
     return arena + plan->offsets[i];
   };
 
-  const long long S = seq_len(c), D = c.hidden, F = c.ffn;
+  // S: the token rows this plan covers (the owned rows of its shard; all of them without
+  // sharding), row0: the first of them; S_all: every row -- the keys and values of all shards
+  const long long S_all = seq_len(c), D = c.hidden, F = c.ffn;
+  int64_t row0_ = 0, rows_ = 0;
+  if (shard_rows(c, plan->shard, &row0_, &rows_)) return XEMA_EINVAL;
+  const long long S = rows_, row0 = row0_;
   const int CA = plan->chunks[0], CB = plan->chunks[1], CC = plan->chunks[2];
   for (int l = 0; l < c.n_blocks; ++l) {
     const xema_block_weights& w = weights[l];
@@ -310,7 +342,7 @@ int xema_plan_bind(xema_plan* plan, void* arena_dev, uint64_t arena_bytes, const
     Op op{};
     op.kind = OP_MOD;
     op.temb = temb; op.w_mod = w.w_mod; op.b_mod = w.b_mod; op.mod = mod;
-    const double Bd = c.batch, Dd = (double)D, Fd = (double)F, Sd = (double)S;
+    const double Bd = c.batch, Dd = (double)D, Fd = (double)F, Sd = (double)S_all;
     auto tag = [&](Op& o, const char* nm, int chunk, double flops, double bytes) {
       std::snprintf(o.name, sizeof(o.name), "%s", nm);
       o.block = l; o.chunk = chunk; o.flops = flops; o.bytes = bytes;
@@ -339,8 +371,10 @@ int xema_plan_bind(xema_plan* plan, void* arena_dev, uint64_t arena_bytes, const
       }
       return pc;
     };
-    // byte offset of (batch b0, row r0) in a full-size [B, S, width] tensor
+    // byte offset of (batch b0, row r0) in a [B, S, width] tensor over the plan's rows, and in the
+    // [B, S_all, 2D] keys-and-values tensor, whose rows are global
     auto at_row = [&](const Piece& pc, long long width, int elem_bytes) { return (pc.b0 * S + pc.r0) * width * elem_bytes; };
+    auto at_kv_row = [&](const Piece& pc) { return (pc.b0 * S_all + row0 + pc.r0) * 2 * D * 2; };
     auto ln_op = [&](const void* in, int f32, void* out, const Piece& pc, int which, const char* nm, int chunk) {
       Op o{};
       o.kind = OP_LN;
@@ -387,18 +421,18 @@ int xema_plan_bind(xema_plan* plan, void* arena_dev, uint64_t arena_bytes, const
       const int n = pc.n;
       uint8_t* h1a = at("h1a", l, ci);
       if (!h1a) return XEMA_EINVAL;
-      uint8_t* kv_pc = kv + at_row(pc, 2 * D, 2);
+      uint8_t* kv_pc = kv + at_kv_row(pc);
       ln_op(hid + at_row(pc, D, 2), 0, h1a, pc, 1, "LN1A", ci);
       // K half: RMSNorm * g_k + RoPE in the GEMM epilogue; the KROPE op of the trace is then
       // a placeholder (the fused kernel touches a subset of what the trace says is live)
-      int rc = gemm_op(h1a, D, n, w_qkv + D * D, D, b_qkv + D, kv_pc, 2 * D, S, nullptr, 0, 0, nullptr,
-                       pc, (int)(2 * D), (int)D, XEMA_EPI_BIAS_NORM_ROPE, "KV", ci, w.g_k, (int)D, (int)pc.r0);
+      int rc = gemm_op(h1a, D, n, w_qkv + D * D, D, b_qkv + D, kv_pc, 2 * D, S_all, nullptr, 0, 0, nullptr,
+                       pc, (int)(2 * D), (int)D, XEMA_EPI_BIAS_NORM_ROPE, "KV", ci, w.g_k, (int)D, (int)(row0 + pc.r0));
       if (rc) return rc;
       Op o{};
       o.kind = OP_FUSED;
       tag(o, "KROPE", ci, 0.0, 0.0);
-      o.rope_x = kv_pc; o.rope_ld = 2 * D; o.rope_batch_rows = S; o.rope_g = w.g_k;
-      o.pos0 = (int)pc.r0; o.rows = n; o.batch = pc.nb;
+      o.rope_x = kv_pc; o.rope_ld = 2 * D; o.rope_batch_rows = S_all; o.rope_g = w.g_k;
+      o.pos0 = (int)(row0 + pc.r0); o.rows = n; o.batch = pc.nb;
       plan->ops.push_back(o);
     }
     // phase B: queries, attention and the gated output projection of every piece
@@ -412,7 +446,7 @@ int xema_plan_bind(xema_plan* plan, void* arena_dev, uint64_t arena_bytes, const
       float* lse = reinterpret_cast<float*>(at("lse", l, ci));
       if (!h1b || !q || !o_t || !lse) return XEMA_EINVAL;
       const uint8_t* hid_pc = hid + at_row(pc, D, 2);
-      const uint8_t* kv_b = kv + pc.b0 * S * 2 * D * 2;          // keys and values of these batch elements
+      const uint8_t* kv_b = kv + pc.b0 * S_all * 2 * D * 2;      // keys and values of these batch elements
       ln_op(hid_pc, 0, h1b, pc, 1, "LN1B", ci);
       // With one piece in both phases LN1B recomputes what LN1A wrote.  When the layout put h1b
       // at h1a's address and nothing was born in between (KROPE allocates nothing, so the only
@@ -437,21 +471,21 @@ int xema_plan_bind(xema_plan* plan, void* arena_dev, uint64_t arena_bytes, const
         }
       }
       int rc = gemm_op(h1b, D, n, w_qkv, D, b_qkv, q, D, n, nullptr, 0, 0, nullptr, pc, (int)D, (int)D,
-                       XEMA_EPI_BIAS_NORM_ROPE, "Q", ci, w.g_q, (int)D, (int)pc.r0);
+                       XEMA_EPI_BIAS_NORM_ROPE, "Q", ci, w.g_q, (int)D, (int)(row0 + pc.r0));
       if (rc) return rc;
       Op o{};
       o.kind = OP_FUSED;
       tag(o, "QROPE", ci, 0.0, 0.0);
-      o.rope_x = q; o.rope_ld = D; o.rope_batch_rows = n; o.rope_g = w.g_q; o.pos0 = (int)pc.r0; o.rows = n;
+      o.rope_x = q; o.rope_ld = D; o.rope_batch_rows = n; o.rope_g = w.g_q; o.pos0 = (int)(row0 + pc.r0); o.rows = n;
       o.batch = pc.nb;
       plan->ops.push_back(o);
       Op a{};
       a.kind = OP_ATTN;
       // q and o once, k and v once per launch, lse
       tag(a, "ATTN", ci, 4.0 * Bd * n * Sd * Dd, 4.0 * Bd * n * Dd + 4.0 * Bd * Sd * Dd + 4.0 * Bd * c.heads * n);
-      a.attn.o = o_t; a.attn.lse = lse; a.attn.batch = pc.nb; a.attn.rows = n; a.attn.keys = (int)S;
+      a.attn.o = o_t; a.attn.lse = lse; a.attn.batch = pc.nb; a.attn.rows = n; a.attn.keys = (int)S_all;
       a.attn.heads = c.heads; a.attn.head_dim = c.head_dim; a.attn.status = status;
-      rc = attn_prepare(&a.attn, q, D, n, kv_b, kv_b + D * 2, 2 * D, S);
+      rc = attn_prepare(&a.attn, q, D, n, kv_b, kv_b + D * 2, 2 * D, S_all);
       if (rc) return rc;
       plan->ops.push_back(a);
       rc = gemm_op(o_t, D, n, w.w_o, D, w.b_o, res + at_row(pc, D, 4), D, S, hid_pc, D, S,
@@ -501,7 +535,10 @@ int xema_forward_host(const xema_plan* plan, const void* hid_in_host, const void
   auto i_in = plan->index.find("hid0"), i_temb = plan->index.find("temb"), i_out = plan->index.find(out_name);
   if (i_in == plan->index.end() || i_temb == plan->index.end() || i_out == plan->index.end()) return XEMA_EINVAL;
   // exact sizes (the planned sizes are rounded up to 256 bytes; the caller's buffers are not)
-  const size_t hid_bytes = (size_t)2 * c.batch * (size_t)seq_len(c) * c.hidden;
+  int64_t own_rows = 0;
+  if (shard_rows(c, plan->shard, nullptr, &own_rows)) return XEMA_EINVAL;
+  if (plan->shard.P != 1) return XEMA_ESTATE;   // a shard's step needs the caller's exchange in the middle
+  const size_t hid_bytes = (size_t)2 * c.batch * (size_t)own_rows * c.hidden;
   const size_t temb_bytes = (size_t)2 * c.batch * c.temb_dim;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   cudaError_t e = cudaMemcpyAsync(plan->arena + plan->offsets[i_in->second], hid_in_host, hid_bytes, cudaMemcpyHostToDevice, st);

@@ -27,11 +27,15 @@ class BlockSession:
     the phases whose trace exceeds the budget) and one count for the whole block; `serialize`
     lets that search split a phase into sub-batches instead of row chunks where the batch allows
     it (temporary serialization).  `axes` gives the split axis per phase for explicit `chunks`.
+    `shard` = (p, P) binds the plan of one sequence-parallel shard (explicit `chunks` only): the
+    session's input and output are then the shard's own token rows, and `forward_sharded` runs the
+    step with the caller's exchange of keys and values in the middle of every block.
     """
 
     def __init__(self, template, weights: Sequence[dict], chunks=None,
                  budget_bytes: Optional[int] = None, max_chunks: int = 64, device="cuda:0",
-                 arena: Optional[torch.Tensor] = None, per_phase: bool = True, axes=None, serialize: bool = False):
+                 arena: Optional[torch.Tensor] = None, per_phase: bool = True, axes=None, serialize: bool = False,
+                 shard=None):
         if not torch.cuda.is_available():
             raise RuntimeError("a CUDA device is required (there is no CPU fallback)")
         self.device = torch.device(device)
@@ -50,7 +54,9 @@ class BlockSession:
             if chunks is None:
                 raise xb.XemaError(xb.XEMA_EBUDGET, search.__name__)
         self.budget_bytes = budget_bytes
-        self.plan = xb.Plan(self.cfg, chunks, axes)
+        if shard is not None and budget_bytes is not None:
+            raise ValueError("a sharded session takes explicit chunks")
+        self.plan = xb.Plan(self.cfg, chunks, axes, shard)
         self.chunks = chunks
         self.phase_chunks = self.plan.phase_chunks
         self.axes = self.plan.axes
@@ -73,7 +79,8 @@ class BlockSession:
         self.arena = arena
         self.status = torch.zeros(1, dtype=torch.int32, device=self.device)
         self.plan.bind(self.arena.data_ptr(), self.arena.numel(), ptrs, self.rope.data_ptr(), self.status.data_ptr())
-        self.seq = template.s_text + template.grid_t * template.grid_h * template.grid_w
+        self.seq_all = template.s_text + template.grid_t * template.grid_h * template.grid_w
+        self.seq = self.plan.rows          # token rows of this session's tensors (all of them unless sharded)
 
     # ---- views into the arena ---------------------------------------------------------
     def view(self, name: str, dtype=torch.int16, shape=None) -> torch.Tensor:
@@ -110,6 +117,27 @@ class BlockSession:
             self.plan.block_forward(s)
         else:
             self.plan.step_forward(s)
+
+    def kv(self, block: int = 0) -> torch.Tensor:
+        """Keys and values of `block`, [B, S, 2D] over ALL token rows (K half first per row)."""
+        t = self.template
+        _, off = self.plan.gather_point(block)
+        n = 2 * t.batch * self.seq_all * 2 * t.hidden
+        return self.arena[off:off + n].view(torch.int16).view(t.batch, self.seq_all, 2 * t.hidden)
+
+    def forward_sharded(self, exchange, stream: Optional[torch.cuda.Stream] = None):
+        """The forward pass of a sequence-parallel shard: for every block, the ops up to its
+        gather point, then `exchange(block)` -- which must leave the other shards' rows of
+        `self.kv(block)` in place, ordered after the enqueued work on `stream` and before what is
+        enqueued next -- then on to the next gather point."""
+        s = (stream or torch.cuda.current_stream(self.device)).cuda_stream
+        at = 0
+        for l in range(self.template.n_blocks):
+            op, _ = self.plan.gather_point(l)
+            self.plan.forward_range(at, op, s)
+            exchange(l)
+            at = op
+        self.plan.forward_range(at, self.plan.n_ops, s)
 
     def capture(self, stream: Optional[torch.cuda.Stream] = None) -> "torch.cuda.CUDAGraph":
         """Records one forward pass into a CUDA graph (every address is static, so the graph
@@ -193,3 +221,16 @@ class BlockSession:
     def staging_bytes(self) -> int:
         t = self.template
         return 2 * (2 * t.batch * self.seq * t.hidden) + 2 * t.batch * t.temb_dim
+
+
+def all_gather_rows(full: torch.Tensor, row_ranges, group=None):
+    """The exchange of sequence parallelism on a [B, S, W] tensor every rank holds in full size:
+    rank r has filled rows row_ranges[r] = (first row, rows) of every batch element; afterwards
+    every rank holds all rows.  One broadcast per (rank, batch element) -- the row ranges differ
+    in size by up to one row, which a plain all-gather of equal parts cannot express -- straight
+    into the tensor itself (for a session: into its own arena); no peer memory is ever read by a
+    kernel.  Works on CPU tensors (gloo) and CUDA tensors (NCCL)."""
+    import torch.distributed as dist
+    for r, (r0, n) in enumerate(row_ranges):
+        for b in range(full.shape[0]):
+            dist.broadcast(full[b, r0:r0 + n], src=dist.get_global_rank(group, r) if group is not None else r, group=group)

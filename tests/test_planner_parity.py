@@ -231,3 +231,42 @@ def test_pressure_ranges_bit_exact():
             assert xb.xema_pressure_ranges(ts, n_ops, budget) == o_arena.pressure_ranges(ts, n_ops, budget)
     with pytest.raises(xb.XemaError):
         xb.xema_pressure_ranges([{"bytes": 256, "birth": 2, "death": 2}], 4, 0)
+
+
+def test_sharded_trace_and_plan_bit_exact():
+    """Sequence-parallel shards: the library's trace, offsets, peak and row ranges equal the
+    oracle's for every shard of several shard counts, chunkings and split axes."""
+    cases = [("tiny", 1, (1, 1, 1), None), ("tiny", 1, (2, 3, 1), None), ("tiny", 2, (1, 2, 2), (0, 1, 1)),
+             ("cogvideox", 1, (1, 1, 2), None), ("flux", 4, (1, 2, 4), (0, 0, 1)), ("step", 1, (1, 1, 2), None)]
+    for name, batch, counts, axes in cases:
+        t = template(name, batch=batch)
+        cfg = xb.make_config(t)
+        for P in (1, 2, 3, 8):
+            if name == "step" and P not in (2, 8):
+                continue
+            for p in range(P):
+                want, want_ops = o_trace.trace(t, counts, axes or (0, 0, 0), shard=(p, P))
+                got, n_ops = xb.xema_trace_sharded(cfg, counts, axes, p, P)
+                assert n_ops == want_ops and len(got) == len(want)
+                for g, w in zip(got, want):
+                    assert all(g[k] == w[k] for k in ("name", "kind", "dtype", "block", "chunk", "bytes", "birth", "death")), (g, w)
+                assert xb.xema_shard_rows(cfg, p, P) == o_trace.shard_rows(t, (p, P))
+                if name == "step" and p not in (0, P - 1):
+                    continue
+                pl = xb.Plan(cfg, counts, axes, shard=(p, P))
+                w_offs, w_peak = o_arena.plan_arena(want)
+                assert [d["offset"] for d in pl.tensors()] == w_offs and pl.peak_bytes == w_peak
+                assert pl.max_live_bytes == o_arena.max_live_bytes(want, want_ops)
+                assert (pl.shard, (pl.row0, pl.rows)) == ((p, P), o_trace.shard_rows(t, (p, P)))
+                ca, cb, cc = counts
+                for l in range(t.n_blocks if name != "step" else 2):
+                    op, off = pl.gather_point(l)
+                    assert op == l * (1 + 3 * ca + 5 * cb + 3 * cc) + 1 + 3 * ca
+                    assert off == pl.tensor("kv%d" % l)[0]
+                pl.close()
+    cfg = xb.make_config(template("tiny"))
+    for bad in ((2, 2), (-1, 2), (0, 0), (0, 289)):
+        with pytest.raises(xb.XemaError):
+            xb.xema_shard_rows(cfg, *bad)
+    with pytest.raises(xb.XemaError):
+        xb.Plan(cfg, (1, 200, 1), shard=(0, 2))            # more chunks than owned rows (144)
