@@ -239,6 +239,18 @@ int xema_plan_mitigation(const xema_plan* plan, xema_mitigation* m);
  * xema_forward_host refuses a sharded plan (XEMA_ESTATE). */
 int xema_plan_create_sharded(const xema_config* cfg, const xema_mitigation* m, int32_t shard, int32_t shards,
                              xema_plan** out);
+/* Debug layout with guard bands (a stand-in for a memory checker): every tensor is laid out as
+ * if it were guard_bytes (a multiple of 256) larger, so the guard_bytes after it -- [offset +
+ * bytes, offset + bytes + guard_bytes) -- belong to no tensor for as long as it lives.  A caller
+ * fills those bytes with a pattern when the tensor is born and checks them after every op until it
+ * dies (tensor lifetimes: xema_plan_tensor_at; one op at a time: xema_forward_range): a kernel
+ * that writes past the end of its own tensor shows up at once, with the op that did it.  The
+ * reported tensor sizes and max-live bytes are the real ones; the peak includes the guards.
+ * Outputs are the same bits as with any other layout. */
+int xema_plan_create_guarded(const xema_config* cfg, const xema_mitigation* m, int32_t shard, int32_t shards,
+                             uint64_t guard_bytes, xema_plan** out);
+/* guard_bytes of the plan (0 for a plan made any other way). */
+uint64_t xema_plan_guard_bytes(const xema_plan* plan);
 /* The plan's shard and the rows it owns (0 of 1 and all rows for an unsharded plan). */
 int xema_plan_shard(const xema_plan* plan, int32_t* shard, int32_t* shards, int64_t* row0, int64_t* rows);
 /* Gather point of block `block`: *first_op = index of the first op of its phase B (every op

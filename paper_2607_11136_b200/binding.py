@@ -25,7 +25,7 @@ EXPORTS = (
     "xema_plan_info", "xema_plan_phase_chunks", "xema_plan_mitigation", "xema_plan_tensor",
     "xema_plan_tensor_at", "xema_plan_bind", "xema_block_forward", "xema_step_forward",
     "xema_block_forward_static",
-    "xema_shard_rows", "xema_trace_sharded", "xema_plan_create_sharded", "xema_plan_shard", "xema_plan_gather_point",
+    "xema_shard_rows", "xema_trace_sharded", "xema_plan_create_sharded", "xema_plan_shard", "xema_plan_gather_point", "xema_plan_create_guarded", "xema_plan_guard_bytes",
     "xema_plan_launch_count", "xema_forward_host", "xema_forward_prefix", "xema_forward_range", "xema_plan_op", "xema_op_mod", "xema_op_ln_modulate",
     "xema_op_rmsnorm_rope", "xema_op_gemm", "xema_op_attention", "xema_strerror",
     "xema_last_cuda_error", "xema_version", "xema_selftest_wait_timeout",
@@ -104,6 +104,8 @@ def lib() -> C.CDLL:
             "xema_trace_sharded": [P(xema_config), P(xema_mitigation), i32, i32, P(xema_tensor), sz, P(sz), P(u32)],
             "xema_shard_rows": [P(xema_config), i32, i32, P(i64), P(i64)],
             "xema_plan_shard": [vp, P(i32), P(i32), P(i64), P(i64)],
+            "xema_plan_create_guarded": [P(xema_config), P(xema_mitigation), i32, i32, u64, P(vp)],
+            "xema_plan_guard_bytes": [vp],
             "xema_plan_gather_point": [vp, i32, P(u32), P(u64)],
             "xema_plan_mitigation": [vp, P(xema_mitigation)],
             "xema_plan_phase_chunks": [vp, P(i32)],
@@ -145,6 +147,7 @@ def lib() -> C.CDLL:
         L.xema_plan_destroy.restype = None
         L.xema_strerror.argtypes = [C.c_int]
         L.xema_strerror.restype = C.c_char_p
+        L.xema_plan_guard_bytes.restype = C.c_uint64
         L.xema_version.argtypes = []
         L.xema_version.restype = C.c_char_p
         _lib = L
@@ -352,13 +355,21 @@ def xema_rope_table(cfg: xema_config) -> np.ndarray:
 class Plan:
     """Owner of an xema_plan handle."""
 
-    def __init__(self, cfg: xema_config, chunks, axes=None, shard=None):
+    def __init__(self, cfg: xema_config, chunks, axes=None, shard=None, guard_bytes: int = 0):
         """chunks: one count (xema_plan_create) or a per-phase triple (xema_plan_create_phases);
         with `axes` (per-phase SPLIT_ROWS / SPLIT_BATCH) xema_plan_create_mitigated; with
-        `shard` = (p, P) xema_plan_create_sharded (the plan of one sequence-parallel shard)."""
+        `shard` = (p, P) xema_plan_create_sharded (the plan of one sequence-parallel shard); with
+        `guard_bytes` xema_plan_create_guarded (debug layout with a guard band after every tensor)."""
         self.cfg = cfg
         self._h = C.c_void_p()
-        if shard is not None:
+        self.guard_bytes = int(guard_bytes)
+        if guard_bytes:
+            c3 = (chunks,) * 3 if isinstance(chunks, int) else chunks
+            m = _mitigation(c3, axes or (SPLIT_ROWS,) * 3)
+            sh = shard or (0, 1)
+            _check(lib().xema_plan_create_guarded(C.byref(cfg), C.byref(m), sh[0], sh[1], guard_bytes, C.byref(self._h)),
+                   "xema_plan_create_guarded")
+        elif shard is not None:
             c3 = (chunks,) * 3 if isinstance(chunks, int) else chunks
             m = _mitigation(c3, axes or (SPLIT_ROWS,) * 3)
             _check(lib().xema_plan_create_sharded(C.byref(cfg), C.byref(m), shard[0], shard[1], C.byref(self._h)),

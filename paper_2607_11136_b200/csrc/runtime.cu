@@ -125,6 +125,7 @@ struct xema_plan {
   int32_t chunks[3];  // key/value, attention, feed-forward phase
   int32_t axes[3];    // XEMA_SPLIT_ROWS or XEMA_SPLIT_BATCH per phase
   Shard shard;        // sequence-parallel shard this plan covers ({0, 1}: the whole sequence)
+  uint64_t guard;     // debug layout: bytes kept free after every tensor (0 in a normal plan)
   std::vector<xema_tensor> tensors;
   std::vector<uint64_t> offsets;
   std::unordered_map<std::string, size_t> index;
@@ -192,7 +193,13 @@ int xema_plan_create_mitigated(const xema_config* cfg, const xema_mitigation* m,
 
 int xema_plan_create_sharded(const xema_config* cfg, const xema_mitigation* m, int32_t shard, int32_t shards,
                              xema_plan** out) {
+  return xema_plan_create_guarded(cfg, m, shard, shards, 0, out);
+}
+
+int xema_plan_create_guarded(const xema_config* cfg, const xema_mitigation* m, int32_t shard, int32_t shards,
+                             uint64_t guard_bytes, xema_plan** out) {
   if (!cfg || !out || !m) return XEMA_EINVAL;
+  if (guard_bytes % 256 || guard_bytes > (1ull << 30)) return XEMA_EINVAL;
   *out = nullptr;
   xema_plan* pl = new (std::nothrow) xema_plan();
   if (!pl) return XEMA_ENOSPC;
@@ -208,9 +215,20 @@ int xema_plan_create_sharded(const xema_config* cfg, const xema_mitigation* m, i
   pl->shard.p = shard;
   pl->shard.P = shards;
   int rc = build_trace(*cfg, chunks, pl->axes, pl->shard, pl->tensors, &pl->n_ops);
+  pl->guard = guard_bytes;
   if (!rc) {
     pl->offsets.assign(pl->tensors.size(), 0);
-    rc = plan_arena(pl->tensors.data(), pl->tensors.size(), pl->offsets.data(), &pl->peak, &pl->live);
+    if (guard_bytes == 0) {
+      rc = plan_arena(pl->tensors.data(), pl->tensors.size(), pl->offsets.data(), &pl->peak, &pl->live);
+    } else {
+      // lay out tensors that are guard_bytes larger than they are: the bytes after every tensor
+      // then belong to nobody for as long as the tensor lives
+      std::vector<xema_tensor> padded(pl->tensors);
+      for (xema_tensor& t : padded) t.bytes += guard_bytes;
+      uint64_t padded_live = 0;
+      rc = plan_arena(padded.data(), padded.size(), pl->offsets.data(), &pl->peak, &padded_live);
+      pl->live = max_live(pl->tensors.data(), pl->tensors.size());
+    }
   }
   if (rc) {
     delete pl;
@@ -255,6 +273,8 @@ int xema_plan_shard(const xema_plan* plan, int32_t* shard, int32_t* shards, int6
   if (shards) *shards = plan->shard.P;
   return shard_rows(plan->cfg, plan->shard, row0, rows);
 }
+
+uint64_t xema_plan_guard_bytes(const xema_plan* plan) { return plan ? plan->guard : 0; }
 
 int xema_plan_gather_point(const xema_plan* plan, int32_t block, uint32_t* first_op, uint64_t* kv_offset) {
   if (!plan || block < 0 || block >= plan->cfg.n_blocks) return XEMA_EINVAL;

@@ -30,12 +30,14 @@ class BlockSession:
     `shard` = (p, P) binds the plan of one sequence-parallel shard (explicit `chunks` only): the
     session's input and output are then the shard's own token rows, and `forward_sharded` runs the
     step with the caller's exchange of keys and values in the middle of every block.
+    `guard_bytes` > 0 binds the debug layout with a guard band after every tensor (explicit
+    `chunks` only); `forward_guarded` then runs op by op and checks the bands.
     """
 
     def __init__(self, template, weights: Sequence[dict], chunks=None,
                  budget_bytes: Optional[int] = None, max_chunks: int = 64, device="cuda:0",
                  arena: Optional[torch.Tensor] = None, per_phase: bool = True, axes=None, serialize: bool = False,
-                 shard=None):
+                 shard=None, guard_bytes: int = 0):
         if not torch.cuda.is_available():
             raise RuntimeError("a CUDA device is required (there is no CPU fallback)")
         self.device = torch.device(device)
@@ -56,7 +58,9 @@ class BlockSession:
         self.budget_bytes = budget_bytes
         if shard is not None and budget_bytes is not None:
             raise ValueError("a sharded session takes explicit chunks")
-        self.plan = xb.Plan(self.cfg, chunks, axes, shard)
+        if guard_bytes and budget_bytes is not None:
+            raise ValueError("a guarded session takes explicit chunks")
+        self.plan = xb.Plan(self.cfg, chunks, axes, shard, guard_bytes)
         self.chunks = chunks
         self.phase_chunks = self.plan.phase_chunks
         self.axes = self.plan.axes
@@ -138,6 +142,41 @@ class BlockSession:
             exchange(l)
             at = op
         self.plan.forward_range(at, self.plan.n_ops, s)
+
+    GUARD_PATTERN = 0xA5
+
+    def _guard(self, d) -> torch.Tensor:
+        g = self.plan.guard_bytes
+        return self.arena[d["offset"] + d["bytes"]:d["offset"] + d["bytes"] + g]
+
+    def forward_guarded(self, stream: Optional[torch.cuda.Stream] = None, exchange=None):
+        """The forward pass one op at a time over the guarded layout: the guard band of a tensor
+        is filled with a pattern just before the op that gives birth to it (for the inputs: now,
+        so call this after set_inputs) and checked after every op for as long as the tensor
+        lives.  Returns the violations as (op index, op name, tensor name, damaged bytes): a
+        kernel that writes past the end of its tensor is caught at the op that did it.  An empty
+        list means every band stayed intact.  `exchange(block)`: as in forward_sharded."""
+        if not self.plan.guard_bytes:
+            raise ValueError("the session was not created with guard_bytes")
+        st = stream or torch.cuda.current_stream(self.device)
+        tensors = self.plan.tensors()
+        gather = {self.plan.gather_point(l)[0]: l for l in range(self.template.n_blocks)} if exchange else {}
+        bad = []
+        with torch.cuda.stream(st):
+            for k in range(self.plan.n_ops):
+                for d in tensors:
+                    if d["birth"] == k:
+                        self._guard(d).fill_(self.GUARD_PATTERN)
+                if k in gather:
+                    exchange(gather[k])
+                self.plan.forward_range(k, k + 1, st.cuda_stream)
+                name = self.plan.op(k)["name"]
+                for d in tensors:
+                    if d["birth"] <= k < d["death"]:
+                        n = int((self._guard(d) != self.GUARD_PATTERN).sum().item())
+                        if n:
+                            bad.append((k, name, d["name"], n))
+        return bad
 
     def capture(self, stream: Optional[torch.cuda.Stream] = None) -> "torch.cuda.CUDAGraph":
         """Records one forward pass into a CUDA graph (every address is static, so the graph

@@ -423,3 +423,53 @@ def test_forward_replayed_from_a_cuda_graph(tiny_case):
     t_eager = (time.perf_counter() - t0) / 200
     print("tiny block: %.1f us per replayed graph, %.1f us eager" % (t_graph * 1e6, t_eager * 1e6))
     s.check_status()
+
+
+@pytest.mark.parametrize("name,chunks", [("tiny", (1, 2, 3)), ("cogvideox", (1, 1, 2))])
+def test_guard_bands_between_arena_neighbours_stay_intact(name, chunks):
+    """Debug layout with 4 KiB kept free after every tensor (the stand-in for a memory checker):
+    run op by op, the band after every live tensor keeps its pattern after every op; the output
+    has the bits of the ordinary layout.  The checker itself is shown to see a damaged band."""
+    t = template(name)
+    w = make_block_weights(t, 0)
+    x, temb = make_activations(t)
+    s = BlockSession(t, [w], chunks=chunks)
+    s.set_inputs(x, temb)
+    s.forward()
+    want = s.output_bits().copy()
+    G = 4096
+    g = BlockSession(t, s.weights, chunks=chunks, guard_bytes=G)
+    tensors = g.plan.tensors()
+    assert g.plan.guard_bytes == G and g.plan.max_live_bytes == s.plan.max_live_bytes
+    assert s.plan.peak_bytes < g.plan.peak_bytes <= s.plan.peak_bytes + G * len(tensors)
+    # no two tensors that live together come closer than the guard
+    for i, a in enumerate(tensors):
+        for b in tensors[i + 1:]:
+            if a["birth"] < b["death"] and b["birth"] < a["death"]:
+                lo, hi = (a, b) if a["offset"] < b["offset"] else (b, a)
+                assert lo["offset"] + lo["bytes"] + G <= hi["offset"], (lo["name"], hi["name"])
+    g.set_inputs(x, temb)
+    assert g.forward_guarded() == []
+    assert np.array_equal(g.output_bits(), want)
+    g.check_status()
+    # negative control: a byte written into the band behind the block input is reported by the
+    # first op (the input is live from op 0) and by every op up to the input's last use
+    g.set_inputs(x, temb)
+    hid0 = next(d for d in tensors if d["name"] == "hid0")
+    real_fill = torch.Tensor.fill_
+    damaged = {"done": False}
+
+    def fill_then_damage(self_, value):
+        out = real_fill(self_, value)
+        if not damaged["done"] and self_.data_ptr() == g.arena.data_ptr() + hid0["offset"] + hid0["bytes"]:
+            self_[7] = 0
+            damaged["done"] = True
+        return out
+
+    torch.Tensor.fill_ = fill_then_damage
+    try:
+        bad = g.forward_guarded()
+    finally:
+        torch.Tensor.fill_ = real_fill
+    assert damaged["done"] and bad and bad[0][:1] == (0,) and all(b[2] == "hid0" and b[3] == 1 for b in bad)
+    assert len(bad) == hid0["death"]
