@@ -13,6 +13,8 @@
 //             other accumulator
 // A row's result depends only on (row, N, K): the K loop always runs in the same order and the
 // tile shape is chosen from N alone, so outputs are bit-identical however rows are chunked.
+#include <type_traits>
+
 #include "kernels.h"
 #include "sm100.cuh"
 
@@ -121,6 +123,81 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, int b, int r
   }
 }
 
+// The two gated epilogues for one 32-column chunk of a warp's 32 rows, with coalesced global
+// accesses.  In the accumulator a thread owns a row, so a warp-wide 16-byte access would touch 32
+// different rows -- 32 separate lines per instruction, eight store instructions and four to eight
+// residual loads per chunk; the load/store unit then takes longer over a tile's epilogue (30 000
+// cycles measured) than the tensor pipe over the next tile's main loop (22 000).  Here the accumulator
+// goes through a per-warp shared-memory tile (rows padded to 36 floats) and comes back
+// transposed: eight lanes cover the 32 columns of one row, a warp instruction covers four whole
+// rows, and residual, gate and output are accessed a full row segment at a time.
+constexpr int STAGE_LD = 36;                         // floats per staged row (16-byte aligned, conflict-light)
+constexpr int STAGE_FLOATS = 32 * STAGE_LD;          // per warp
+template <int EPI>
+struct GatedResid {
+  typename std::conditional<EPI == XEMA_EPI_GATE_RES_F32, uint2, float4>::type x[8];
+  float4 gate;   // of the lane's four columns
+  uint2 bias;    // four bf16
+};
+// Requests what a lane needs for one chunk besides the accumulator: the residual values of its
+// four columns in eight rows, and the gate and bias of those columns.
+template <int EPI>
+__device__ __forceinline__ void gated_load_resid(const GemmParams& p, int b, int row0, int n0, int lane, GatedResid<EPI>& rs) {
+  const int c4 = (lane & 7) * 4;
+  const int rbase = row0 + (lane >> 3);
+  rs.gate = __ldg(reinterpret_cast<const float4*>(p.gate + (size_t)b * p.gate_stride + n0 + c4));
+  rs.bias = __ldg(reinterpret_cast<const uint2*>(p.bias + n0 + c4));
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int row = rbase + 4 * i;
+    if (row < p.rows) {
+      const size_t rrow = ((size_t)b * p.resid_batch_rows + row) * p.ldr + n0 + c4;
+      if constexpr (EPI == XEMA_EPI_GATE_RES_F32)
+        rs.x[i] = __ldg(reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(p.resid) + rrow));
+      else
+        rs.x[i] = __ldg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(p.resid) + rrow));
+    }
+  }
+}
+template <int EPI>
+__device__ __forceinline__ void epilogue_chunk_gated(const GemmParams& p, int b, int row0, int n0, const uint32_t (&r)[32],
+                                                     float* stage, int lane, const GatedResid<EPI>& rs) {
+  {
+    // the raw accumulator row of this thread into the tile
+    uint4* sp = reinterpret_cast<uint4*>(stage + lane * STAGE_LD);
+#pragma unroll
+    for (int q = 0; q < 8; ++q) sp[q] = make_uint4(r[4 * q], r[4 * q + 1], r[4 * q + 2], r[4 * q + 3]);
+  }
+  __syncwarp();
+  const int c4 = (lane & 7) * 4;                     // this lane's four columns of the chunk
+  const float4 g = rs.gate;
+  const float4 bs = make_float4(bf16_lo(rs.bias.x), bf16_hi(rs.bias.x), bf16_lo(rs.bias.y), bf16_hi(rs.bias.y));
+  const int rbase = row0 + (lane >> 3);
+  float4 v[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const float4 a = *reinterpret_cast<const float4*>(stage + (4 * i + (lane >> 3)) * STAGE_LD + c4);
+    v[i] = make_float4(a.x + bs.x, a.y + bs.y, a.z + bs.z, a.w + bs.w);
+  }
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int row = rbase + 4 * i;
+    if (row < p.rows) {
+      const size_t orow = ((size_t)b * p.out_batch_rows + row) * p.ldo + n0 + c4;
+      if constexpr (EPI == XEMA_EPI_GATE_RES_F32) {
+        *reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + orow) =
+            make_float4(fmaf(g.x, v[i].x, bf16_lo(rs.x[i].x)), fmaf(g.y, v[i].y, bf16_hi(rs.x[i].x)),
+                        fmaf(g.z, v[i].z, bf16_lo(rs.x[i].y)), fmaf(g.w, v[i].w, bf16_hi(rs.x[i].y)));
+      } else {
+        *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(p.out) + orow) =
+            make_uint2(pack_bf16x2(fmaf(g.x, v[i].x, rs.x[i].x), fmaf(g.y, v[i].y, rs.x[i].y)),
+                       pack_bf16x2(fmaf(g.z, v[i].z, rs.x[i].z), fmaf(g.w, v[i].w, rs.x[i].w)));
+      }
+    }
+  }
+  __syncwarp();                                      // the tile is free for the next chunk
+}
+
 // One head (DH columns starting at n0) of this thread's row: acc + bias, RMSNorm over the head,
 // gain, rotation of adjacent pairs by the token's angles, bf16 store.
 template <int DH>
@@ -167,8 +244,11 @@ __device__ __forceinline__ void epilogue_head_norm_rope(const GemmParams& p, int
 }
 
 // The finished BN-wide accumulator row of one thread (TMEM address t_addr) -> global memory.
+// `stage`: the warp's shared-memory tile for the coalesced form of the gated epilogues, or null
+// (every thread then reads and writes its own row directly).
 template <int BN, int EPI>
-__device__ __forceinline__ void epilogue_row(const GemmParams& p, int b, int row, int n_base, uint32_t t_addr) {
+__device__ __forceinline__ void epilogue_row(const GemmParams& p, int b, int row, int n_base, uint32_t t_addr,
+                                             float* stage = nullptr) {
   if constexpr (EPI == XEMA_EPI_BIAS_NORM_ROPE) {
     // head by head; heads at or beyond norm_cols (the V half of a KV product) get the bias only
 #pragma unroll 1
@@ -188,6 +268,29 @@ __device__ __forceinline__ void epilogue_row(const GemmParams& p, int b, int row
       }
     }
   } else {
+    if constexpr (EPI == XEMA_EPI_GATE_RES_F32 || EPI == XEMA_EPI_GATE_RES_BF16) {
+      if (stage) {
+        // coalesced form; the residual of chunk c+1 is requested before chunk c is worked on, and
+        // all loads of a chunk are in flight together (one memory round trip per chunk, covered)
+        const int lane = threadIdx.x & 31;
+        const int row0 = row - lane;
+        GatedResid<EPI> ra, rb;
+        gated_load_resid<EPI>(p, b, row0, n_base, lane, ra);
+#pragma unroll 1
+        for (int ch = 0; ch < BN / 32; ch += 2) {
+          uint32_t r[32];
+          gated_load_resid<EPI>(p, b, row0, n_base + (ch + 1) * 32, lane, rb);
+          tmem_ld32(t_addr + ch * 32, r);
+          tmem_ld_wait();
+          epilogue_chunk_gated<EPI>(p, b, row0, n_base + ch * 32, r, stage, lane, ra);
+          if (ch + 2 < BN / 32) gated_load_resid<EPI>(p, b, row0, n_base + (ch + 2) * 32, lane, ra);
+          tmem_ld32(t_addr + (ch + 1) * 32, r);
+          tmem_ld_wait();
+          epilogue_chunk_gated<EPI>(p, b, row0, n_base + (ch + 1) * 32, r, stage, lane, rb);
+        }
+        return;
+      }
+    }
 #pragma unroll 1
     for (int ch = 0; ch < BN / 32; ++ch) {
       uint32_t r[32];
@@ -385,7 +488,8 @@ constexpr int PAIR_BN = 256;
 constexpr int PAIR_STAGES = 6;
 constexpr int PAIR_B_HALF_BYTES = (PAIR_BN / 2) * BK * 2;
 constexpr int PAIR_STAGE_BYTES = A_TILE_BYTES + PAIR_B_HALF_BYTES;
-constexpr int PAIR_SMEM_BYTES = 1024 + PAIR_STAGES * PAIR_STAGE_BYTES + 256;
+constexpr int PAIR_STAGE_TILE_BYTES = 4 * STAGE_FLOATS * 4;      // one transposition tile per epilogue warp
+constexpr int PAIR_SMEM_BYTES = 1024 + PAIR_STAGES * PAIR_STAGE_BYTES + 256 + PAIR_STAGE_TILE_BYTES;
 constexpr int PAIR_TMEM_COLS = 2 * PAIR_BN;
 // Limit of one drain wait after a give-up (about 50 ms): long enough for any copy in flight,
 // short enough that six of them in a row stay far below the limit of a regular wait.
@@ -540,7 +644,8 @@ gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
       tc_fence_after();
       const int row = (c.mt * 2 + (int)rank) * BM + quad * 32 + lane;
       const uint32_t t_addr = tmem_base + ((uint32_t)(quad * 32) << 16) + acc * PAIR_BN;
-      epilogue_row<PAIR_BN, EPI>(p, c.b, row, c.nt * PAIR_BN, t_addr);
+      epilogue_row<PAIR_BN, EPI>(p, c.b, row, c.nt * PAIR_BN, t_addr,
+                                 reinterpret_cast<float*>(bar_base + 256) + quad * STAGE_FLOATS);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(mapa_shared(smem_u32(&tmem_empty[acc]), 0));
