@@ -397,6 +397,8 @@ typedef struct xema_gemm_args {
                            normalise and rotate (D for a K|V product, N for a Q product)   */
   int32_t rope_pos0;    /* token index of row 0: row i uses table row rope_pos0 + i        */
   float rms_eps;
+  float norm_out_scale; /* the normalised, rotated heads are multiplied by this before the
+                           rounding to bf16; 0 means 1 (the other columns are never scaled)   */
   const void* norm_gain; /* device bf16 [head_dim]                                          */
   const float* rope;     /* device fp32 [tokens][head_dim/2][cos, sin]                      */
 } xema_gemm_args;
@@ -407,11 +409,18 @@ int xema_op_gemm(const xema_gemm_args* args, void* status_dev, void* stream);
  * q: device bf16, row (b,i) at (b*q_batch_rows + i)*ldq, head h at feature h*head_dim.
  * k, v: device bf16, key (b,j) at (b*kv_batch_rows + j)*ldkv (k and v are separate base
  * pointers into the same rows).  o: device bf16 [B,rows,heads*head_dim] contiguous.
- * lse: device fp32 [B,heads,rows] or NULL. */
+ * lse: device fp32 [B,heads,rows] or NULL.
+ * q_scale (> 0): what q k^T is multiplied by to give exponents to base 2.  For a plain q pass
+ * log2(e) / sqrt(head_dim).  Pass 1 if q was already multiplied by that -- the block does this in
+ * the fused epilogue of the Q projection (norm_out_scale), where it costs no extra rounding: the
+ * head_dim 64 kernel takes the exponents straight from the tensor core.  Given any other q_scale
+ * that kernel multiplies its copy of the q tiles in shared memory first, which rounds q to bf16 a
+ * second time (relative 2^-9 per element; visible where |q k^T| / sqrt(head_dim) reaches the
+ * hundreds). */
 int xema_op_attention(const void* q, int64_t ldq, int64_t q_batch_rows, const void* k, const void* v,
                       int64_t ldkv, int64_t kv_batch_rows, void* o, float* lse, int32_t batch,
-                      int32_t rows, int32_t keys, int32_t heads, int32_t head_dim, void* status_dev,
-                      void* stream);
+                      int32_t rows, int32_t keys, int32_t heads, int32_t head_dim, float q_scale,
+                      void* status_dev, void* stream);
 
 /* ---- allocator plug-in ------------------------------------------------------------------ */
 /* The paper's run-time mechanism for code that is not this library's own kernels (section

@@ -75,7 +75,8 @@ class xema_gemm_args(C.Structure):
                 ("gate", C.c_void_p), ("gate_stride", C.c_int64),
                 ("batch", C.c_int32), ("rows", C.c_int32), ("N", C.c_int32), ("K", C.c_int32),
                 ("epilogue", C.c_int32), ("head_dim", C.c_int32), ("norm_cols", C.c_int32),
-                ("rope_pos0", C.c_int32), ("rms_eps", C.c_float), ("norm_gain", C.c_void_p),
+                ("rope_pos0", C.c_int32), ("rms_eps", C.c_float), ("norm_out_scale", C.c_float),
+                ("norm_gain", C.c_void_p),
                 ("rope", C.c_void_p)]
 
 
@@ -135,7 +136,7 @@ def lib() -> C.CDLL:
             "xema_op_ln_modulate": [vp, i32, i64, vp, vp, vp, i64, i32, i32, i32, C.c_float, vp],
             "xema_op_rmsnorm_rope": [vp, i64, i64, vp, vp, i32, i32, i32, i32, i32, C.c_float, vp],
             "xema_op_gemm": [P(xema_gemm_args), vp, vp],
-            "xema_op_attention": [vp, i64, i64, vp, vp, i64, i64, vp, vp, i32, i32, i32, i32, i32, vp, vp],
+            "xema_op_attention": [vp, i64, i64, vp, vp, i64, i64, vp, vp, i32, i32, i32, i32, i32, C.c_float, vp, vp],
             "xema_last_cuda_error": [],
             "xema_selftest_wait_timeout": [vp, i64, vp, vp],
         }
@@ -515,7 +516,17 @@ def xema_op_gemm(status=None, stream=0, **kw):
     _check(lib().xema_op_gemm(C.byref(a), status, stream), "xema_op_gemm")
 
 
+def exponent_scale(head_dim: int) -> float:
+    """log2(e) / sqrt(head_dim) as the float32 the library uses: q k^T times this = exponents to base 2."""
+    import numpy as np
+    return float(np.float32(1.4426950408889634) / np.sqrt(np.float32(head_dim)))
+
+
 def xema_op_attention(q, ldq, q_batch_rows, k, v, ldkv, kv_batch_rows, o, lse, batch, rows, keys, heads, head_dim,
-                      status=None, stream=0):
+                      status=None, stream=0, q_scale=None):
+    """q_scale: None for a plain q (log2(e) / sqrt(head_dim) is passed), 1.0 for a q that was
+    already multiplied by exponent_scale(head_dim)."""
+    if q_scale is None:
+        q_scale = exponent_scale(head_dim)
     _check(lib().xema_op_attention(q, ldq, q_batch_rows, k, v, ldkv, kv_batch_rows, o, lse, batch, rows, keys, heads,
-                                   head_dim, status, stream), "xema_op_attention")
+                                   head_dim, q_scale, status, stream), "xema_op_attention")

@@ -409,8 +409,8 @@ static int launch_attention_t(const AttnLaunch& a, cudaStream_t stream) {
   p.rows = a.rows;
   p.keys = a.keys;
   p.heads = a.heads;
-  p.scale = 1.0f / sqrtf((float)DH);
-  p.scale_log2 = p.scale * 1.4426950408889634f;
+  p.scale_log2 = a.q_scale;                         // scores times this = exponents to base 2
+  p.scale = a.q_scale * 0.6931471805599453f;        // ... and times this = natural exponents (for lse)
   p.status = a.status;
   dim3 grid((a.rows + ATT_BM - 1) / ATT_BM, a.heads, a.batch);
   kern<<<grid, ATT_THREADS, Cfg::SMEM_BYTES, stream>>>(a.map_q, a.map_k, a.map_v, p);

@@ -25,7 +25,14 @@
 //     exponential polynomial an argument outside its range, is flagged, and its CTA runs two more
 //     sweeps: one that only takes the true row maximum, one that repeats the pass with that
 //     maximum as the reference of the flagged rows and with the polynomial's arguments clamped.
-//     Rows that were not flagged repeat exactly what they did before, bit for bit.
+//     Rows that were not flagged repeat exactly what they did before, bit for bit;
+//   * the scores leave the tensor core as finished exponents.  q arrives multiplied by
+//     log2(e) / sqrt(64) (the Q projection's epilogue does that before its one rounding to bf16;
+//     a plain q is multiplied here, in shared memory), and from the second key block on the
+//     contraction has a fifth 16-wide step over [-reference, 0, ...] x [1, 0, ...] -- two small
+//     constant-shaped operands next to Q and K in shared memory, the reference (as a bf16
+//     number) written there by the row's thread -- so S = q k - reference and a softmax thread's
+//     work per pair of scores is the exponential, one packed add for the row sum and one pack.
 //
 //   warp 0      TMA producer: both Q tiles once, then K and V tiles through a ring of stages
 //   warp 1      owns TMEM; converged warp, one elected lane issues S(j+1) of a tile as soon as
@@ -58,7 +65,9 @@ constexpr int STAGES = 4;
 constexpr int OFF_Q = 0;
 constexpr int OFF_K = OFF_Q + TILES * Q_TILE_BYTES;
 constexpr int OFF_V = OFF_K + STAGES * KV_TILE_BYTES;
-constexpr int OFF_XCH = OFF_V + STAGES * KV_TILE_BYTES;      // float [2 slots][TILES][2 halves][BM]
+constexpr int OFF_QX = OFF_V + STAGES * KV_TILE_BYTES;       // per tile: 128 rows x 128 B, column 0 = -reference
+constexpr int OFF_KX = OFF_QX + TILES * Q_TILE_BYTES;        // 128 keys x 128 B, column 0 = 1
+constexpr int OFF_XCH = OFF_KX + KV_TILE_BYTES;              // float [2 slots][TILES][2 halves][BM]
 constexpr int OFF_BAR = OFF_XCH + 2 * TILES * 2 * BM * 4;
 constexpr int SMEM_BYTES = OFF_BAR + 512;
 constexpr int TMEM_COLS = 512;   // per tile 256: S [0,128), P [128,192), O [192,256)
@@ -87,20 +96,22 @@ __device__ __forceinline__ f32x2 exp2_poly_unclamped(f32x2 x2) {
                      __uint_as_float(__float_as_uint(p2.y) + (__float_as_uint(t2.y) << 23)));
 }
 
-// p = 2^(s * c + nm) for 16 consecutive score columns: 8 packed bf16x2 words, the values added
+// p = 2^(s + nm) for 16 consecutive score columns: 8 packed bf16x2 words, the values added
 // into four packed partial sums.  POLY_NUM of every POLY_DEN column pairs (fixed positions)
 // evaluate 2^x as a polynomial on the FMA pipe, the others on the MUFU.  The polynomial is only
 // valid for arguments in [-125, 126].  SAFE = false: it is used as it is and `poly_abs` collects
 // the largest magnitude handed to it, for the caller to check afterwards.  SAFE = true:
 // arguments are clamped from below first (2^-125 stands in for zero); wherever the unclamped
 // form was valid the result has the same bits.
-template <bool SAFE>
-__device__ __forceinline__ void exp16(const float (&s)[16], f32x2 c2, f32x2 nm2, uint32_t (&pk)[8], f32x2 (&ls2)[4],
+template <bool SAFE, bool SHIFT>
+__device__ __forceinline__ void exp16(const float (&s)[16], f32x2 nm2, uint32_t (&pk)[8], f32x2 (&ls2)[4],
                                       float& poly_abs) {
 #pragma unroll
   for (int t = 0; t < 16; t += 2) {
     const int pair = t >> 1;
-    f32x2 e2 = fma_f32x2(pack_f32x2(s[t], s[t + 1]), c2, nm2);
+    // SHIFT: the scores still need the row's reference taken off (first key block); otherwise
+    // they come out of the tensor core as exponents already
+    f32x2 e2 = SHIFT ? add_f32x2(pack_f32x2(s[t], s[t + 1]), nm2) : pack_f32x2(s[t], s[t + 1]);
     float e0, e1;
     if ((pair % POLY_DEN) < POLY_NUM) {
       if (SAFE) {
@@ -152,7 +163,7 @@ struct Attn64Params {
   __nv_bfloat16* o;
   float* lse;
   int batch, rows, keys, heads;
-  float scale, scale_log2;
+  float q_scale;      // q k^T times this = exponents to base 2 (1: q arrives already multiplied)
   unsigned int* status;
 };
 
@@ -171,7 +182,8 @@ attention_dh64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
   uint64_t* p_full = bars + 21;    // [TILES] P(j) of the tile is complete in TMEM
   uint64_t* pv_done = bars + 23;   // [TILES] O += P(j) V(j) has finished
   uint64_t* xch_bar = bars + 25;   // [TILES * 4] the two warps that share 32 rows exchange a value
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 33);
+  uint64_t* q_ready = bars + 33;   // the Q tiles are scaled and the extension operands are set up
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 34);
   volatile uint32_t* abort_flag = tmem_slot + 1;
   volatile uint32_t* danger_any = tmem_slot + 2;
   volatile float* xch = reinterpret_cast<volatile float*>(smem + OFF_XCH);
@@ -200,6 +212,7 @@ attention_dh64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
       mbar_init(&pv_done[t], 1);
     }
     for (int i = 0; i < TILES * 4; ++i) mbar_init(&xch_bar[i], 64);
+    mbar_init(q_ready, 32 * SOFTMAX_WARPS);
     *abort_flag = 0;
     *danger_any = 0;
     fence_mbar_init();
@@ -298,14 +311,19 @@ attention_dh64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
       constexpr uint32_t idesc_s = idesc_bf16_f32(BM, BN, false, false);
       const uint64_t q_desc0 = smem_desc_sw128(smem_u32(smem + OFF_Q), 16, 1024);
       const uint64_t k_desc0 = smem_desc_sw128(smem_u32(smem + OFF_K), 16, 1024);
-      auto issue_s = [&](int t, uint64_t k_desc) {   // elected lane only
+      const uint64_t qx_desc0 = smem_desc_sw128(smem_u32(smem + OFF_QX), 16, 1024);
+      const uint64_t kx_desc = smem_desc_sw128(smem_u32(smem + OFF_KX), 16, 1024);
+      // with_ref: one more 16-wide step of the contraction, over [-reference, 0, ...] x [1, 0, ...]:
+      // the scores arrive with the row's reference already taken off
+      auto issue_s = [&](int t, uint64_t k_desc, bool with_ref) {   // elected lane only
         const uint32_t d = tmem_base + t * TM_TILE;
         const uint64_t q_desc = q_desc0 + (uint64_t)(t * (Q_TILE_BYTES >> 4));
 #pragma unroll
         for (int k = 0; k < DH / 16; ++k) mma_ss(d, q_desc + (uint64_t)(2 * k), k_desc + (uint64_t)(2 * k), idesc_s, k != 0);
+        if (with_ref) mma_ss(d, qx_desc0 + (uint64_t)(t * (Q_TILE_BYTES >> 4)), kx_desc, idesc_s, 1);
         mma_commit(&s_full[t]);
       };
-      if (ok && sweep == 0) ok = mbar_wait_warp(q_full, 0, abort_flag);
+      if (ok && sweep == 0) ok = mbar_wait_warp(q_full, 0, abort_flag) && mbar_wait_warp(q_ready, 0, abort_flag);
       // S(0) of both tiles at once (the softmax threads are done with the previous sweep's scores:
       // the sweeps are separated by a CTA-wide barrier); S(j+1) of a tile as soon as its threads
       // hold S(j) in registers
@@ -320,7 +338,7 @@ attention_dh64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
           }
           tc_fence_after();
           if (elect_one()) {
-            issue_s(t, k_desc);
+            issue_s(t, k_desc, j > 0 && !scores_only);
             if (t == TILES - 1) mma_commit(&k_empty[k_st]);
           }
           __syncwarp();
@@ -357,7 +375,49 @@ attention_dh64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
       }
     } else if (ok) {
       // ---------------- softmax ----------------
-      const f32x2 c2 = pack_f32x2(p.scale_log2, p.scale_log2);
+      // where a row's reference sits in the extension operand of its tile (128-byte swizzle:
+      // the 16-byte chunk holding column 0 of row r is chunk r % 8 of the row)
+      __nv_bfloat16* ref_slot = reinterpret_cast<__nv_bfloat16*>(smem + OFF_QX + tile * Q_TILE_BYTES + r * 128 + (r & 7) * 16);
+      auto publish_ref = [&]() {
+        // the reference as a bf16 number (any value near the maximum serves, as long as the same
+        // one is used everywhere), negated, into column 0 of the extension operand
+        const __nv_bfloat16 q = __float2bfloat16_rn(m_ref);
+        m_ref = __bfloat162float(q);
+        neg_ref = -m_ref;
+        if (half == 0) *ref_slot = __float2bfloat16_rn(neg_ref);
+        fence_proxy_async_smem();
+      };
+      if (sweep == 0) {
+        // One-time set-up by the 512 softmax threads: the extension operands (zeros, and a one in
+        // column 0 of every key row), and and, for a q that does not arrive in exponent
+        // units, its tiles multiplied so that scores are exponents to base 2.
+        const int ts = threadIdx.x - 96;
+        uint4* zx = reinterpret_cast<uint4*>(smem + OFF_QX);
+        for (int i = ts; i < (TILES * Q_TILE_BYTES + KV_TILE_BYTES) / 16; i += 32 * SOFTMAX_WARPS) {
+          uint4 v = make_uint4(0u, 0u, 0u, 0u);
+          const int k = i - TILES * Q_TILE_BYTES / 16;       // 16-byte chunk index inside the key operand
+          if (k >= 0 && (k & 7) == ((k >> 3) & 7)) v.x = 0x3F80u;   // bf16 1.0 in column 0 of key row k / 8
+          zx[i] = v;
+        }
+        if (p.q_scale != 1.f) {
+          // a plain q: its tiles are multiplied here (a second rounding to bf16)
+          ok = mbar_wait_warp(q_full, 0, abort_flag);
+          if (ok) {
+            uint4* qv = reinterpret_cast<uint4*>(smem + OFF_Q);
+            for (int i = ts; i < TILES * Q_TILE_BYTES / 16; i += 32 * SOFTMAX_WARPS) {
+              uint4 v = qv[i];
+              uint32_t* w = reinterpret_cast<uint32_t*>(&v);
+#pragma unroll
+              for (int e = 0; e < 4; ++e) w[e] = pack_bf16x2(bf16_lo(w[e]) * p.q_scale, bf16_hi(w[e]) * p.q_scale);
+              qv[i] = v;
+            }
+          }
+        }
+        if (ok) {
+          fence_proxy_async_smem();
+          mbar_arrive(q_ready);
+        }
+      }
       auto u16 = [](float(&a)[16]) -> uint32_t(&)[16] { return *reinterpret_cast<uint32_t(*)[16]>(&a[0]); };
       auto u32 = [](float(&a)[32]) -> uint32_t(&)[32] { return *reinterpret_cast<uint32_t(*)[32]>(&a[0]); };
       // the largest score of this thread's half of block j
@@ -384,10 +444,7 @@ attention_dh64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
           m_true = fmaxf(m_true, mine);
         }
       } else {
-        if (sweep == 2 && danger_row) {
-          m_ref = m_true;
-          neg_ref = -m_ref * p.scale_log2;
-        }
+        // (the new reference of a flagged row was published at the end of the second sweep)
         if (sweep == 0) {
           // the row's reference exponent: the largest score of its first key block
           ok = mbar_wait_warp(&s_full[tile], sfull_ph, abort_flag);
@@ -395,7 +452,7 @@ attention_dh64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
             tc_fence_after();
             const float mine = half_max(0);
             m_ref = fmaxf(mine, exchange(mine));
-            neg_ref = -m_ref * p.scale_log2;
+            publish_ref();
           }
         }
         const f32x2 nm2 = pack_f32x2(neg_ref, neg_ref);
@@ -429,17 +486,17 @@ attention_dh64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
           tmem_ld_wait_on(u16(b1));
           tmem_ld_wait_on(u16(b2));
           if (MASKED && valid < 16) mask_tail16(b0, valid);
-          exp16<SAFE>(b0, c2, nm2, pk8(0), ls2, poly_abs);
+          exp16<SAFE, FIRST>(b0, nm2, pk8(0), ls2, poly_abs);
           tmem_ld16(s_tmem + 48, u16(b0));
           if (MASKED && valid < 32) mask_tail16(b1, valid - 16);
-          exp16<SAFE>(b1, c2, nm2, pk8(1), ls2, poly_abs);
+          exp16<SAFE, FIRST>(b1, nm2, pk8(1), ls2, poly_abs);
           tmem_ld_wait_on(u16(b0));
           tc_fence_before();
           mbar_arrive(&s_free[tile]);                       // S(j) is in registers: S(j+1) may land
           if (MASKED && valid < 48) mask_tail16(b2, valid - 32);
-          exp16<SAFE>(b2, c2, nm2, pk8(2), ls2, poly_abs);
+          exp16<SAFE, FIRST>(b2, nm2, pk8(2), ls2, poly_abs);
           if (MASKED) mask_tail16(b0, valid - 48);
-          exp16<SAFE>(b0, c2, nm2, pk8(3), ls2, poly_abs);
+          exp16<SAFE, FIRST>(b0, nm2, pk8(3), ls2, poly_abs);
           if (!FIRST) {
             if (!mbar_peek(&pv_done[tile], pv_ph)) ok = mbar_wait_warp(&pv_done[tile], pv_ph, abort_flag);
             pv_ph ^= 1;
@@ -479,7 +536,13 @@ attention_dh64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
         danger_row = (exchange(danger ? 1.f : 0.f) != 0.f) || danger;
         if (danger_row) *danger_any = 1;
       }
-      if (ok && sweep == 1) m_true = fmaxf(m_true, exchange(m_true));
+      if (ok && sweep == 1) {
+        m_true = fmaxf(m_true, exchange(m_true));
+        if (danger_row) {
+          m_ref = m_true;
+          publish_ref();
+        }
+      }
     }
     // every role is done with this sweep; the softmax threads' flags are visible after the barrier
     tc_fence_before();
@@ -507,7 +570,7 @@ attention_dh64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
                             pack_bf16x2(__uint_as_float(o[8 * q + 2]) * inv_l, __uint_as_float(o[8 * q + 3]) * inv_l),
                             pack_bf16x2(__uint_as_float(o[8 * q + 4]) * inv_l, __uint_as_float(o[8 * q + 5]) * inv_l),
                             pack_bf16x2(__uint_as_float(o[8 * q + 6]) * inv_l, __uint_as_float(o[8 * q + 7]) * inv_l));
-      if (p.lse && half == 0) p.lse[((size_t)b * p.heads + h) * p.rows + row] = fmaf(m_ref, p.scale, logf(l_row));
+      if (p.lse && half == 0) p.lse[((size_t)b * p.heads + h) * p.rows + row] = fmaf(m_ref, 0.6931471805599453f, logf(l_row));
     }
   }
 
@@ -530,8 +593,7 @@ int launch_attention_dh64(const AttnLaunch& a, cudaStream_t stream) {
   p.rows = a.rows;
   p.keys = a.keys;
   p.heads = a.heads;
-  p.scale = 0.125f;
-  p.scale_log2 = p.scale * 1.4426950408889634f;
+  p.q_scale = a.q_scale;
   p.status = a.status;
   dim3 grid((a.rows + TILES * BM - 1) / (TILES * BM), a.heads, a.batch);
   attention_dh64_kernel<<<grid, THREADS, SMEM_BYTES, stream>>>(a.map_q, a.map_k, a.map_v, p);

@@ -52,7 +52,7 @@ struct GemmParams {
   const __nv_bfloat16* norm_gain;   // [head_dim]
   const float* rope;                // [token][head_dim/2][cos, sin]
   int rope_pos0, head_dim, norm_cols;
-  float rms_eps;
+  float rms_eps, norm_out_scale;
 };
 
 __device__ __forceinline__ float gelu_tanh_f(float z) {
@@ -219,7 +219,7 @@ __device__ __forceinline__ void epilogue_head_norm_rope(const GemmParams& p, int
 #pragma unroll
     for (int t = 0; t < 8; ++t) ss = fmaf(v[8 * q + t], v[8 * q + t], ss);
   }
-  const float rstd = rsqrtf(ss * (1.f / DH) + p.rms_eps);
+  const float rstd = rsqrtf(ss * (1.f / DH) + p.rms_eps) * p.norm_out_scale;
   const float4* rp = reinterpret_cast<const float4*>(p.rope + (size_t)(p.rope_pos0 + row) * DH);
   uint4* op = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.out) +
                                        ((size_t)b * p.out_batch_rows + row) * p.ldo + n0);
@@ -689,6 +689,7 @@ static GemmParams make_params(const GemmLaunch& g) {
   p.head_dim = g.head_dim;
   p.norm_cols = g.norm_cols;
   p.rms_eps = g.rms_eps;
+  p.norm_out_scale = g.norm_out_scale > 0.f ? g.norm_out_scale : 1.f;
   return p;
 }
 

@@ -77,6 +77,7 @@ struct GemmLaunch {
   const float* rope;
   int rope_pos0, head_dim, norm_cols;
   float rms_eps;
+  float norm_out_scale;   // the normalised, rotated heads are multiplied by this before rounding (1 = as they are)
 };
 // Fills map_a / map_w / block_n from plain pointers.
 int gemm_prepare(GemmLaunch* g, const void* a, long long lda, long long a_batch_rows, const void* w, long long ldw);
@@ -90,6 +91,9 @@ struct AttnLaunch {
   void* o;             // bf16 [batch][rows][heads*dh]
   float* lse;          // fp32 [batch][heads][rows] or null
   int batch, rows, keys, heads, head_dim;
+  // what q k^T is multiplied by to give exponents to base 2: log2(e) / sqrt(head_dim) for a plain
+  // q, 1 if q was already multiplied by that (as the fused epilogue of the Q projection does)
+  float q_scale;
   unsigned int* status;
 };
 int attn_prepare(AttnLaunch* a, const void* q, long long ldq, long long q_batch_rows, const void* k, const void* v,

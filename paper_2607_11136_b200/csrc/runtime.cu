@@ -4,6 +4,7 @@
 #include <cuda_bf16.h>
 
 #include <algorithm>
+#include <cmath>
 #include <cstdio>
 #include <cstring>
 #include <new>
@@ -411,13 +412,13 @@ int xema_plan_bind(xema_plan* plan, void* arena_dev, uint64_t arena_bytes, const
                        const void* bias, void* out, long long ldo, long long out_batch_rows, const void* resid,
                        long long ldr, long long resid_batch_rows, const float* gate, const Piece& pc, int N, int K,
                        int epi, const char* nm, int chunk, const void* norm_gain = nullptr, int norm_cols = 0,
-                       int pos0 = 0) -> int {
+                       int pos0 = 0, float norm_out_scale = 1.f) -> int {
       const int rows = pc.n;
       const double Bd = (double)pc.nb;
       Op o{};
       o.kind = OP_GEMM;
       o.gemm.norm_gain = norm_gain; o.gemm.rope = rope_dev; o.gemm.rope_pos0 = pos0; o.gemm.head_dim = c.head_dim;
-      o.gemm.norm_cols = norm_cols; o.gemm.rms_eps = c.rms_eps;
+      o.gemm.norm_cols = norm_cols; o.gemm.rms_eps = c.rms_eps; o.gemm.norm_out_scale = norm_out_scale;
       {
         const double out_b = (epi == XEMA_EPI_GATE_RES_F32) ? 4.0 : 2.0;
         const double res_b = (epi == XEMA_EPI_GATE_RES_F32) ? 2.0 : (epi == XEMA_EPI_GATE_RES_BF16 ? 4.0 : 0.0);
@@ -455,6 +456,10 @@ int xema_plan_bind(xema_plan* plan, void* arena_dev, uint64_t arena_bytes, const
       o.pos0 = (int)(row0 + pc.r0); o.rows = n; o.batch = pc.nb;
       plan->ops.push_back(o);
     }
+    // The queries leave their projection already multiplied by log2(e) / sqrt(head_dim), inside the
+    // epilogue that rounds them to bf16 (one rounding, as before): the attention's scores are then
+    // exponents to base 2 as they come out of the tensor core.
+    const float q_scale = 1.4426950408889634f / std::sqrt((float)c.head_dim);
     // phase B: queries, attention and the gated output projection of every piece
     for (int ci = 0; ci < CB; ++ci) {
       const Piece pc = piece_of(1, ci);
@@ -491,7 +496,7 @@ int xema_plan_bind(xema_plan* plan, void* arena_dev, uint64_t arena_bytes, const
         }
       }
       int rc = gemm_op(h1b, D, n, w_qkv, D, b_qkv, q, D, n, nullptr, 0, 0, nullptr, pc, (int)D, (int)D,
-                       XEMA_EPI_BIAS_NORM_ROPE, "Q", ci, w.g_q, (int)D, (int)(row0 + pc.r0));
+                       XEMA_EPI_BIAS_NORM_ROPE, "Q", ci, w.g_q, (int)D, (int)(row0 + pc.r0), q_scale);
       if (rc) return rc;
       Op o{};
       o.kind = OP_FUSED;
@@ -504,7 +509,7 @@ int xema_plan_bind(xema_plan* plan, void* arena_dev, uint64_t arena_bytes, const
       // q and o once, k and v once per launch, lse
       tag(a, "ATTN", ci, 4.0 * Bd * n * Sd * Dd, 4.0 * Bd * n * Dd + 4.0 * Bd * Sd * Dd + 4.0 * Bd * c.heads * n);
       a.attn.o = o_t; a.attn.lse = lse; a.attn.batch = pc.nb; a.attn.rows = n; a.attn.keys = (int)S_all;
-      a.attn.heads = c.heads; a.attn.head_dim = c.head_dim; a.attn.status = status;
+      a.attn.heads = c.heads; a.attn.head_dim = c.head_dim; a.attn.status = status; a.attn.q_scale = 1.f;
       rc = attn_prepare(&a.attn, q, D, n, kv_b, kv_b + D * 2, 2 * D, S_all);
       if (rc) return rc;
       plan->ops.push_back(a);
@@ -637,7 +642,7 @@ int xema_op_gemm(const xema_gemm_args* a, void* status_dev, void* stream) {
   g.gate = a->gate; g.gate_stride = a->gate_stride;
   g.batch = a->batch; g.rows = a->rows; g.N = a->N; g.K = a->K; g.epilogue = a->epilogue;
   g.norm_gain = a->norm_gain; g.rope = a->rope; g.rope_pos0 = a->rope_pos0; g.head_dim = a->head_dim;
-  g.norm_cols = a->norm_cols; g.rms_eps = a->rms_eps;
+  g.norm_cols = a->norm_cols; g.rms_eps = a->rms_eps; g.norm_out_scale = a->norm_out_scale;
   g.status = static_cast<unsigned int*>(status_dev);
   int rc = gemm_prepare(&g, a->a, a->lda, a->a_batch_rows, a->w, a->ldw);
   if (rc) return rc;
@@ -646,9 +651,11 @@ int xema_op_gemm(const xema_gemm_args* a, void* status_dev, void* stream) {
 
 int xema_op_attention(const void* q, int64_t ldq, int64_t q_batch_rows, const void* k, const void* v, int64_t ldkv,
                       int64_t kv_batch_rows, void* o, float* lse, int32_t batch, int32_t rows, int32_t keys,
-                      int32_t heads, int32_t head_dim, void* status_dev, void* stream) {
+                      int32_t heads, int32_t head_dim, float q_scale, void* status_dev, void* stream) {
+  if (!(q_scale > 0.f)) return XEMA_EINVAL;
   AttnLaunch a{};
   a.o = o; a.lse = lse; a.batch = batch; a.rows = rows; a.keys = keys; a.heads = heads; a.head_dim = head_dim;
+  a.q_scale = q_scale;
   a.status = static_cast<unsigned int*>(status_dev);
   int rc = attn_prepare(&a, q, ldq, q_batch_rows, k, v, ldkv, kv_batch_rows);
   if (rc) return rc;

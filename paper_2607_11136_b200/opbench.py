@@ -51,7 +51,8 @@ def main():
 
     if a.op == "attention":
         D = a.heads * a.head_dim
-        q = _randn_bf16((B, a.rows, D), 1.0, gen)
+        # q in exponent units (as the block's Q projection delivers it): N(0,1) times log2(e) / sqrt(head_dim)
+        q = _randn_bf16((B, a.rows, D), xb.exponent_scale(a.head_dim), gen)
         kv = _randn_bf16((B, a.keys, 2 * D), 1.0, gen)
         o = torch.empty_like(q)
         lse = torch.empty(B, a.heads, a.rows, dtype=torch.float32, device="cuda")
@@ -59,7 +60,7 @@ def main():
         def run():
             xb.xema_op_attention(q.data_ptr(), D, a.rows, kv.data_ptr(), kv.data_ptr() + 2 * D, 2 * D, a.keys,
                                  o.data_ptr(), lse.data_ptr(), B, a.rows, a.keys, a.heads, a.head_dim,
-                                 status=status.data_ptr(), stream=stream)
+                                 status=status.data_ptr(), stream=stream, q_scale=1.0)
         flops = 4.0 * B * a.rows * a.keys * D
         nbytes = 4.0 * B * a.rows * D + 4.0 * B * a.keys * D + 4.0 * B * a.heads * a.rows
     elif a.op == "gemm":

@@ -7,7 +7,7 @@ import torch
 
 from oracle import block as ob
 from paper_2607_11136_b200 import binding as xb
-from xema_inputs import template
+from xema_inputs import bf16_bits, bits_to_f64, template
 
 from gpu_util import DEV, assert_bf16_close, assert_close, from_dev_bf16, rand_bf16, to_dev
 
@@ -169,16 +169,25 @@ def test_gemm_rows_are_chunk_invariant():
     assert torch.equal(full[:, r0:r0 + n], part)
 
 
+def _exponent_units(q_f32, dh):
+    """What the Q projection's fused epilogue hands the attention: q multiplied by
+    log2(e) / sqrt(dh) in float32 and rounded to bf16 once.  Returns (bits, the exact float64 q
+    those bits stand for)."""
+    c = np.float32(xb.exponent_scale(dh))
+    bits = bf16_bits(q_f32.astype(np.float32) * c)
+    return bits, bits_to_f64(bits) / np.float64(c)
+
+
 def _attention_case(rng, B, rows, keys, H, dh, q_scale=1.0):
     D = H * dh
-    qb, qf = rand_bf16(rng, (B, rows, D), q_scale)
+    qb, qf = _exponent_units(rng.standard_normal((B, rows, D), dtype=np.float32) * np.float32(q_scale), dh)
     kvb, kvf = rand_bf16(rng, (B, keys, 2 * D))
     q_dev, kv_dev = to_dev(qb), to_dev(kvb)
     o = torch.full((B, rows, D), 0x7FC0, dtype=torch.int16, device=DEV)
     lse = torch.full((B, H, rows), float("nan"), dtype=torch.float32, device=DEV)
     status = torch.zeros(1, dtype=torch.int32, device=DEV)
     xb.xema_op_attention(q_dev.data_ptr(), D, rows, kv_dev.data_ptr(), kv_dev.data_ptr() + D * 2, 2 * D, keys,
-                         o.data_ptr(), lse.data_ptr(), B, rows, keys, H, dh, status=status.data_ptr())
+                         o.data_ptr(), lse.data_ptr(), B, rows, keys, H, dh, status=status.data_ptr(), q_scale=1.0)
     _sync_status(status)
     ref_o = np.empty((B, rows, H, dh))
     ref_l = np.empty((B, H, rows))
@@ -207,6 +216,31 @@ def test_attention_peaked_scores():
     got_o, ref_o, got_l, ref_l = _attention_case(rng, 1, 256, 1500, 2, 64, q_scale=6.0)
     assert_bf16_close(got_o, ref_o, "attention peaked", atol_rms=1.5e-2, cos=0.9999)
     assert np.abs(got_l - ref_l).max() < 5e-3 * max(1.0, np.abs(ref_l).max())
+
+
+@pytest.mark.parametrize("dh", [64, 128])
+def test_attention_with_a_plain_q(dh):
+    """A q that was not multiplied beforehand: the library is told the scale.  The head_dim 64
+    kernel then multiplies its copy of the q tiles itself, which rounds q a second time (relative
+    2^-9 per element), so the bound is the element-wise bf16 bound with twice the slack."""
+    rng = np.random.default_rng(44 + dh)
+    B, rows, keys, H = 1, 200, 700, 2
+    D = H * dh
+    qb, qf = rand_bf16(rng, (B, rows, D))
+    kvb, kvf = rand_bf16(rng, (B, keys, 2 * D))
+    q_dev, kv_dev = to_dev(qb), to_dev(kvb)
+    o = torch.full((B, rows, D), 0x7FC0, dtype=torch.int16, device=DEV)
+    lse = torch.full((B, H, rows), float("nan"), dtype=torch.float32, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    xb.xema_op_attention(q_dev.data_ptr(), D, rows, kv_dev.data_ptr(), kv_dev.data_ptr() + D * 2, 2 * D, keys,
+                         o.data_ptr(), lse.data_ptr(), B, rows, keys, H, dh, status=status.data_ptr())
+    _sync_status(status)
+    got = from_dev_bf16(o)
+    for h in range(H):
+        ref_o, ref_l = ob.attention_head(qf[0, :, h * dh:(h + 1) * dh], kvf[0, :, h * dh:(h + 1) * dh],
+                                         kvf[0, :, D + h * dh:D + (h + 1) * dh], 1 / math.sqrt(dh))
+        assert_bf16_close(got[0, :, h * dh:(h + 1) * dh], ref_o, ("plain q", dh, h), atol_rms=3e-2, cos=0.9999)
+        assert np.abs(lse.cpu().numpy()[0, h] - ref_l).max() < 4e-3
 
 
 def test_attention_rows_are_chunk_invariant():
@@ -279,15 +313,14 @@ def test_attention_scores_growing_along_the_keys(dh):
     for h in range(H):
         q[0, :, h * dh:(h + 1) * dh] = u[h] * 40.0 + 0.3 * rng.standard_normal((rows, dh))
         kv[0, :, h * dh:(h + 1) * dh] = u[h] * ramp * 60.0 + 0.3 * rng.standard_normal((keys, dh))
-    from xema_inputs import bf16_bits, bits_to_f64
-    qb, kvb = bf16_bits(q.astype(np.float32)), bf16_bits(kv.astype(np.float32))
-    qf, kvf = bits_to_f64(qb), bits_to_f64(kvb)
+    (qb, qf), kvb = _exponent_units(q, dh), bf16_bits(kv.astype(np.float32))
+    kvf = bits_to_f64(kvb)
     q_dev, kv_dev = to_dev(qb), to_dev(kvb)
     o = torch.zeros(B, rows, D, dtype=torch.int16, device=DEV)
     lse = torch.zeros(B, H, rows, dtype=torch.float32, device=DEV)
     status = torch.zeros(1, dtype=torch.int32, device=DEV)
     xb.xema_op_attention(q_dev.data_ptr(), D, rows, kv_dev.data_ptr(), kv_dev.data_ptr() + D * 2, 2 * D, keys,
-                         o.data_ptr(), lse.data_ptr(), B, rows, keys, H, dh, status=status.data_ptr())
+                         o.data_ptr(), lse.data_ptr(), B, rows, keys, H, dh, status=status.data_ptr(), q_scale=1.0)
     _sync_status(status)
     got = from_dev_bf16(o)
     for h in range(H):
