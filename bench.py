@@ -75,17 +75,18 @@ def whole_job_tflops(flops_per_replica: float, world: int, ms: float) -> float:
 
 
 # DRAM traffic of one attention launch (dram__bytes_read.sum + dram__bytes_write.sum under ncu, see
-# profiles/attention_dh64_rows2222_keys17776_h48.md).  Measured inside this bench at the full 17776 query
-# rows: 421.4 MB (329.6 read + 91.7 written; q is still in L2 from the Q projection).  Measured alone at
-# 2222 rows: 254.4 MB, of which k and v (4*S*D bytes, independent of the number of query rows) are read
-# once and the rest scales with the query rows; other row counts are scaled from that capture.
+# profiles/attention_dh64_rows2222_keys17776_h48.md).  Captured inside this bench at the full 17776
+# query rows: 422.9 MB (329.0 read + 93.9 written; algorithmic 440.3 -- q is still in L2 from the Q
+# projection).  Captured alone at 2222 rows: 266.6 MB (algorithmic 246.2), of which k and v (4*S*D
+# bytes, independent of the number of query rows) are read once and the rest scales with the query
+# rows; other row counts are scaled from that capture.  Not measured in the timed run.
 def attention_traffic_bytes(t, rows: int) -> float:
     if (t.seq, t.hidden, t.head_dim) != (17776, 3072, 64):
         return None
     if rows == t.seq:
-        return 421.4e6
+        return 422.9e6
     kv = 4.0 * t.seq * t.hidden
-    return kv + (254.4e6 - kv) * rows / 2222.0
+    return kv + (266.6e6 - kv) * rows / 2222.0
 
 
 class ClockSampler:
