@@ -519,7 +519,8 @@ def main():
         # are NOT part of the budget, so it is the extra, not the value.
         "e2e": {"value": whole_job_tflops(flops, world, e2e_serial_ms), "unit": UNIT, "ms_per_step": e2e_serial_ms,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "how": "xema_forward_host: host-to-device copy, forward, device-to-host copy in order on one stream",
+                "how": "xema_forward_host: pinned host -> arena, forward, arena -> pinned host; the output of a finished "
+                       "feed-forward piece is copied out while the next piece runs (plan-owned copy stream)",
                 "device_bytes": sess.plan.peak_bytes, "fits_budget": budget is None or sess.plan.peak_bytes <= budget,
                 "pipelined": {"value": whole_job_tflops(flops, world, e2e_ms), "ms_per_step": e2e_ms,
                               "how": "BlockSession.run_pipelined: copies of neighbouring steps overlap compute",

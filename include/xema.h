@@ -286,7 +286,13 @@ int xema_step_forward(const xema_plan* plan, void* stream);
  * Enqueues on `stream`: a host-to-device copy of hid_in_host [B,S,D] bf16 and temb_host [B,Dt]
  * bf16 into their arena slots, all n_blocks blocks, and a device-to-host copy of the output
  * hidden state into hid_out_host [B,S,D] bf16.  The arena is the one given to xema_plan_bind;
- * nothing else on the device is touched or allocated.  The host buffers are the caller's and
+ * no other device memory is touched or allocated.  Where the first block's key/value phase or
+ * the last block's feed-forward phase runs in more than one piece, the copies of all pieces but
+ * one go through a second stream owned by the plan (created at the first such call, destroyed
+ * with the plan) and are ordered against `stream` by events in both directions: the input of
+ * piece c + 1 arrives while piece c is worked on, the output of piece c leaves while piece
+ * c + 1 is worked on, and `stream` does not pass the call before the last copy has finished.
+ * The results do not depend on it.  The host buffers are the caller's and
  * must stay valid until the stream has passed the call; they should be page-locked (the copies
  * of pageable memory are staged by the CUDA runtime and may block the calling thread).  Does
  * not synchronise.  XEMA_ESTATE if the plan is unbound, XEMA_ECUDA if a copy or launch is

@@ -136,6 +136,15 @@ struct xema_plan {
   uint8_t* arena;     // as given to xema_plan_bind
   const float* rope;
   std::vector<Op> ops;
+  // xema_forward_host: a second stream and one event per piece of the first and last phase, so
+  // that the copies of one piece overlap the launches of its neighbours (made at the first call;
+  // concurrent calls on one plan share the arena and are the caller's error anyway)
+  mutable cudaStream_t copy_stream = nullptr;
+  mutable std::vector<cudaEvent_t> copy_events;
+  ~xema_plan() {
+    for (cudaEvent_t e : copy_events) cudaEventDestroy(e);
+    if (copy_stream) cudaStreamDestroy(copy_stream);
+  }
 };
 
 static int issue(const xema_plan* pl, const Op& op, cudaStream_t st) {
@@ -550,6 +559,17 @@ int xema_step_forward(const xema_plan* plan, void* stream) {
   return run_ops(plan, 0, plan->ops.size(), stream);
 }
 
+// One piece of a [B, rows, D] bf16 tensor (rows [r0, r0 + rows) of `batch` consecutive batch
+// elements, the first at `dev`) between the arena and the host copy of the whole tensor.
+static cudaError_t copy_piece(uint8_t* tensor_dev, uint8_t* tensor_host, const uint8_t* dev, int batch, int rows,
+                              long long row_elems, long long batch_rows, bool to_host, cudaStream_t st) {
+  const size_t off = (size_t)(dev - tensor_dev), pitch = (size_t)batch_rows * row_elems * 2,
+               width = (size_t)rows * row_elems * 2;
+  if (to_host)
+    return cudaMemcpy2DAsync(tensor_host + off, pitch, tensor_dev + off, pitch, width, batch, cudaMemcpyDeviceToHost, st);
+  return cudaMemcpy2DAsync(tensor_dev + off, pitch, tensor_host + off, pitch, width, batch, cudaMemcpyHostToDevice, st);
+}
+
 int xema_forward_host(const xema_plan* plan, const void* hid_in_host, const void* temb_host, void* hid_out_host,
                       void* stream) {
   if (!plan || !hid_in_host || !temb_host || !hid_out_host) return XEMA_EINVAL;
@@ -566,19 +586,96 @@ int xema_forward_host(const xema_plan* plan, const void* hid_in_host, const void
   const size_t hid_bytes = (size_t)2 * c.batch * (size_t)own_rows * c.hidden;
   const size_t temb_bytes = (size_t)2 * c.batch * c.temb_dim;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-  cudaError_t e = cudaMemcpyAsync(plan->arena + plan->offsets[i_in->second], hid_in_host, hid_bytes, cudaMemcpyHostToDevice, st);
-  if (e == cudaSuccess)
-    e = cudaMemcpyAsync(plan->arena + plan->offsets[i_temb->second], temb_host, temb_bytes, cudaMemcpyHostToDevice, st);
-  if (e != cudaSuccess) {
-    t_last_cuda_error = (int)e;
+  uint8_t* in_dev = plan->arena + plan->offsets[i_in->second];
+  uint8_t* out_dev = plan->arena + plan->offsets[i_out->second];
+  uint8_t* in_host = static_cast<uint8_t*>(const_cast<void*>(hid_in_host));
+  uint8_t* out_host = static_cast<uint8_t*>(hid_out_host);
+  const std::vector<Op>& ops = plan->ops;
+  const size_t n = ops.size();
+  cudaError_t e = cudaSuccess;
+  auto fail = [&](cudaError_t err) {
+    t_last_cuda_error = (int)err;
     return XEMA_ECUDA;
+  };
+
+  // The pieces of the first block's key/value phase read the input piece by piece (LN1A of piece c
+  // reads the rows of piece c only), and the pieces of the last block's feed-forward phase finish
+  // the output piece by piece (FFN2 of piece c).  With more than one piece in either phase the
+  // copies run on a second stream, ordered by events: the input of piece c + 1 arrives while
+  // piece c is worked on, the output of piece c leaves while piece c + 1 is worked on.  Bits do
+  // not depend on it.  With one piece the copy is a plain one on the caller's stream.
+  std::vector<size_t> in_ops, out_ops;      // LN1A launches of block 0, FFN2 launches of the last block
+  for (size_t i = 0; i < n; ++i) {
+    if (ops[i].kind == OP_LN && ops[i].block == 0 && !std::strcmp(ops[i].name, "LN1A")) in_ops.push_back(i);
+    if (ops[i].kind == OP_GEMM && ops[i].block == c.n_blocks - 1 && !std::strcmp(ops[i].name, "FFN2")) out_ops.push_back(i);
   }
-  int rc = run_ops(plan, 0, plan->ops.size(), stream);
-  if (rc) return rc;
-  e = cudaMemcpyAsync(hid_out_host, plan->arena + plan->offsets[i_out->second], hid_bytes, cudaMemcpyDeviceToHost, st);
-  if (e != cudaSuccess) {
-    t_last_cuda_error = (int)e;
-    return XEMA_ECUDA;
+  const bool row_major_out = !out_ops.empty() && ops[out_ops[0]].gemm.ldo == c.hidden;
+  const bool split_in = in_ops.size() > 1, split_out = out_ops.size() > 1 && row_major_out;
+  const size_t n_events = (split_in ? in_ops.size() : 0) + (split_out ? out_ops.size() : 0) + 1;
+  if (split_in || split_out) {
+    if (!plan->copy_stream && (e = cudaStreamCreateWithFlags(&plan->copy_stream, cudaStreamNonBlocking)) != cudaSuccess)
+      return fail(e);
+    while (plan->copy_events.size() < n_events) {
+      cudaEvent_t ev;
+      if ((e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming)) != cudaSuccess) return fail(e);
+      plan->copy_events.push_back(ev);
+    }
+  }
+  size_t next_event = 0;
+  cudaStream_t cs = plan->copy_stream;
+
+  // ---- input
+  if ((e = cudaMemcpyAsync(plan->arena + plan->offsets[i_temb->second], temb_host, temb_bytes, cudaMemcpyHostToDevice, st)) != cudaSuccess)
+    return fail(e);
+  std::vector<cudaEvent_t> in_ready(in_ops.size(), nullptr);
+  if (!split_in) {
+    if ((e = cudaMemcpyAsync(in_dev, in_host, hid_bytes, cudaMemcpyHostToDevice, st)) != cudaSuccess) return fail(e);
+  } else {
+    // the copy stream starts where the caller's stream stands (the arena may still be in use by
+    // work enqueued before this call)
+    cudaEvent_t start = plan->copy_events[next_event++];
+    if ((e = cudaEventRecord(start, st)) != cudaSuccess || (e = cudaStreamWaitEvent(cs, start, 0)) != cudaSuccess) return fail(e);
+    for (size_t k = 0; k < in_ops.size(); ++k) {
+      const Op& o = ops[in_ops[k]];
+      e = copy_piece(in_dev, in_host, static_cast<const uint8_t*>(o.ln_in), o.batch, o.rows, c.hidden, o.ln_in_batch_rows,
+                     false, k == 0 ? st : cs);
+      if (e != cudaSuccess) return fail(e);
+      if (k > 0) {
+        in_ready[k] = plan->copy_events[next_event++];
+        if ((e = cudaEventRecord(in_ready[k], cs)) != cudaSuccess) return fail(e);
+      }
+    }
+  }
+
+  // ---- launches, with the waits for input pieces and the copies of finished output pieces
+  size_t k_in = 0, k_out = 0;
+  for (size_t i = 0; i < n; ++i) {
+    if (split_in && k_in < in_ops.size() && i == in_ops[k_in]) {
+      if (in_ready[k_in] && (e = cudaStreamWaitEvent(st, in_ready[k_in], 0)) != cudaSuccess) return fail(e);
+      ++k_in;
+    }
+    int rc = issue(plan, ops[i], st);
+    if (rc) return rc;
+    if (split_out && k_out < out_ops.size() && i == out_ops[k_out]) {
+      const Op& o = ops[i];
+      const bool last = (k_out + 1 == out_ops.size());
+      if (!last) {
+        cudaEvent_t ev = plan->copy_events[next_event++];
+        if ((e = cudaEventRecord(ev, st)) != cudaSuccess || (e = cudaStreamWaitEvent(cs, ev, 0)) != cudaSuccess) return fail(e);
+      }
+      e = copy_piece(out_dev, out_host, static_cast<const uint8_t*>(o.gemm.out), o.gemm.batch, o.gemm.rows, c.hidden,
+                     o.gemm.out_batch_rows, true, last ? st : cs);
+      if (e != cudaSuccess) return fail(e);
+      ++k_out;
+    }
+  }
+  if (!split_out) {
+    if ((e = cudaMemcpyAsync(out_host, out_dev, hid_bytes, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return fail(e);
+  }
+  if (split_in || split_out) {
+    // the caller's stream ends after everything the copy stream was given
+    cudaEvent_t ev = plan->copy_events[next_event++];
+    if ((e = cudaEventRecord(ev, cs)) != cudaSuccess || (e = cudaStreamWaitEvent(st, ev, 0)) != cudaSuccess) return fail(e);
   }
   return XEMA_OK;
 }

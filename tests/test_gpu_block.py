@@ -275,12 +275,42 @@ def test_bounded_wait_gives_up_and_reports():
     assert_close(bits_to_f64(s.output_bits()), ref, "block after a timed-out wait")
 
 
-def test_forward_host_equals_arena_forward(tiny_case):
-    """xema_forward_host (pinned host buffers in and out, copies and launches on one stream)
-    returns the bits of set_inputs / forward / output_bits, twice in a row, and allocates
-    nothing on the device."""
+def test_forward_host_two_batched_blocks_in_pieces():
+    """Two blocks, batch 2: row pieces (each piece = the same rows of both batch elements, a
+    strided copy) and sub-batches in the first and the last phase; bits of the arena forward."""
+    t = template("tiny", batch=2).with_(n_blocks=2)
+    ws = [make_block_weights(t, l) for l in range(2)]
+    x, temb = make_activations(t)
+    stream = torch.cuda.current_stream().cuda_stream
+    want = None
+    for chunks, axes in (((1, 1, 1), None), ((3, 1, 2), None), ((2, 2, 2), (1, 0, 1)), ((2, 1, 3), (0, 0, 0))):
+        s = BlockSession(t, ws, chunks=chunks, axes=axes)
+        s.set_inputs(x, temb)
+        s.forward()
+        got = s.output_bits().copy()
+        if want is None:
+            want = got
+        assert np.array_equal(got, want)
+        x_h = torch.from_numpy(x.view(np.int16)).pin_memory()
+        t_h = torch.from_numpy(temb.view(np.int16)).pin_memory()
+        y_h = torch.zeros_like(x_h).pin_memory()
+        for _ in range(2):
+            y_h.zero_()
+            s.arena.fill_(0x7F)
+            s.plan.forward_host(x_h.data_ptr(), t_h.data_ptr(), y_h.data_ptr(), stream)
+            torch.cuda.synchronize()
+            assert np.array_equal(y_h.numpy().view(np.uint16), want), (chunks, axes)
+        s.check_status()
+
+
+@pytest.mark.parametrize("chunks", [(1, 1, 2), (3, 2, 3), (1, 1, 1)])
+def test_forward_host_equals_arena_forward(tiny_case, chunks):
+    """xema_forward_host (pinned host buffers in and out; with several pieces in the first or the
+    last phase their copies overlap the neighbouring pieces' launches through the plan's own
+    copy stream) returns the bits of set_inputs / forward / output_bits, three times in a row,
+    and allocates no device memory after its first call."""
     t, w, x, temb, ref = tiny_case
-    s = BlockSession(t, [w], chunks=(1, 1, 2))
+    s = BlockSession(t, [w], chunks=chunks)
     s.set_inputs(x, temb)
     s.forward()
     want = s.output_bits().copy()
@@ -288,13 +318,16 @@ def test_forward_host_equals_arena_forward(tiny_case):
     t_h = torch.from_numpy(temb.view(np.int16)).pin_memory()
     y_h = torch.zeros_like(x_h).pin_memory()
     stream = torch.cuda.current_stream().cuda_stream
-    torch.cuda.synchronize()
-    free0, _ = torch.cuda.mem_get_info()
-    for _ in range(2):
+    free0 = None
+    for _ in range(3):
         y_h.zero_()
+        # scribble over the arena: every input byte the forward reads must come from the host copy
+        s.arena.fill_(0x7F)
         s.plan.forward_host(x_h.data_ptr(), t_h.data_ptr(), y_h.data_ptr(), stream)
         torch.cuda.synchronize()
         assert np.array_equal(y_h.numpy().view(np.uint16), want)
+        if free0 is None:
+            free0, _ = torch.cuda.mem_get_info()     # the first call may create the copy stream
     free1, _ = torch.cuda.mem_get_info()
     assert free1 == free0
     s.check_status()
