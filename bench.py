@@ -119,6 +119,10 @@ class ClockSampler:
         try:
             self.nvml, self.handle = self._nvml_handle()
             self.sm_max = float(self.nvml.nvmlDeviceGetMaxClockInfo(self.handle, self.nvml.NVML_CLOCK_SM))
+            try:
+                self.power_limit = self.nvml.nvmlDeviceGetEnforcedPowerLimit(self.handle) / 1000.0   # read-only
+            except Exception:
+                self.power_limit = None
             self.thread = threading.Thread(target=self._poll, daemon=True)
             self.thread.start()
             return
@@ -156,6 +160,7 @@ class ClockSampler:
             reasons = sorted({name for s in self.samples for bit, name in self.NVML_REASONS if s[2] & bit})
             return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_min_mhz": min(sm) if sm else None,
                     "sm_max_mhz": self.sm_max, "power_w_max": max((s[1] for s in self.samples), default=None),
+                    "power_limit_w": self.power_limit,
                     "samples": len(sm), "source": "nvml, 5 ms period", "reasons": reasons}
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no clock source available"]}
@@ -421,11 +426,14 @@ def main():
     TENSOR_OPS = ("KV", "Q", "ATTN", "PROJ", "FFN1", "FFN2")
 
     def regime_of(clk):
-        """A kernel timed while the SM clock holds within 5 % of its maximum is compared with the
-        burst peak; one timed under the power cap with the sustained peak."""
-        if clk.get("sm_mhz") and clk.get("sm_max_mhz") and clk["sm_mhz"] >= 0.95 * clk["sm_max_mhz"]:
-            return "burst"
-        return "sustained"
+        """A kernel is compared with the sustained peak only when it was timed in that regime: the
+        median SM clock more than 5 % below its maximum AND the board's power reading within 10 % of
+        its limit.  A short leg whose clock has begun to fall while the (averaged) power reading is
+        still far below the limit is compared with the burst peak, the larger denominator."""
+        fast = clk.get("sm_mhz") and clk.get("sm_max_mhz") and clk["sm_mhz"] >= 0.95 * clk["sm_max_mhz"]
+        limit = clk.get("power_limit_w") or 1000.0
+        hot = clk.get("power_w_max") is not None and clk["power_w_max"] >= 0.9 * limit
+        return "sustained" if (not fast and hot) else "burst"
 
     def roofline_of(ops_t, clk):
         dom = max(ops_t, key=lambda n: ops_t[n]["ms"])
@@ -440,8 +448,9 @@ def main():
             achieved = d["bytes"] / d["launches"] / per_launch_s / 1e9
             peak, unit, bound = peaks["hbm_gbs"], "GB/s", "hbm"
         r = {"kernel": dom, "bound": bound, "achieved": achieved, "peak": peak, "unit": unit, "frac": achieved / peak,
-             "peak_source": "%s (%s: median SM clock %s of %s MHz)" % (peaks["source"], regime if bound == "tensor" else "copy",
-                                                                      clk.get("sm_mhz"), clk.get("sm_max_mhz")),
+             "peak_source": "%s (%s: median SM clock %s of %s MHz, power up to %s of %s W)" % (
+                 peaks["source"], regime if bound == "tensor" else "copy", clk.get("sm_mhz"), clk.get("sm_max_mhz"),
+                 clk.get("power_w_max"), clk.get("power_limit_w")),
              "ms_per_launch": per_launch_s * 1e3, "launches_per_step": d["launches"]}
         if bound == "tensor":
             r["frac_of_burst"] = achieved / peaks["bf16_burst"]

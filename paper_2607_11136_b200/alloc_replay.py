@@ -12,6 +12,7 @@ request stream an eager framework would issue for this block.  No kernel runs.  
 from __future__ import annotations
 
 import argparse
+import contextlib
 import json
 import os
 import subprocess
@@ -58,25 +59,42 @@ def replay(sequence, rounds: int, device: str = "cuda:0") -> dict:
         _, peak, live = xb.xema_plan_arena(tensors)
         plans.append({"workload": name, "chunks": list(triple), "arena_peak_bytes": peak, "max_live_bytes": live,
                       "tensors": len(tensors), "events": alloc_events(tensors, n_ops), "sizes": [d["bytes"] for d in tensors]})
-    for _ in range(rounds):
-        for p in plans:
-            held = {}
-            for _, kind, i in p["events"]:
-                if kind == "alloc":
-                    held[i] = torch.empty(p["sizes"][i], dtype=torch.uint8, device=device)
-                else:
-                    del held[i]
-            assert not held
+    # The replay allocates from a memory pool of its own: segments that the process already holds
+    # (partly used ones keep their free space through empty_cache) would otherwise take the
+    # replay's tensors without the reserved figure moving at all.
+    pool = None
+    scope = contextlib.nullcontext()
+    if hasattr(torch.cuda, "MemPool") and hasattr(torch.cuda, "use_mem_pool"):
+        try:
+            pool = torch.cuda.MemPool()
+            scope = torch.cuda.use_mem_pool(pool)
+        except RuntimeError:
+            pool, scope = None, contextlib.nullcontext()
+    reserved_peak = 0
+    with scope:
+        for _ in range(rounds):
+            for p in plans:
+                held = {}
+                for _, kind, i in p["events"]:
+                    if kind == "alloc":
+                        held[i] = torch.empty(p["sizes"][i], dtype=torch.uint8, device=device)
+                    else:
+                        del held[i]
+                assert not held
+                if pool is not None:      # a pool's segments stay until it is destroyed: the sum is its peak
+                    reserved_peak = max(reserved_peak, sum(seg["total_size"] for seg in pool.snapshot()))
+    if pool is None:
+        reserved_peak = torch.cuda.max_memory_reserved() - base_reserved
     out = {
         "sequence": [{k: p[k] for k in ("workload", "chunks", "arena_peak_bytes", "max_live_bytes", "tensors")} for p in plans],
         "rounds": rounds,
         "static_arena_bytes": max(p["arena_peak_bytes"] for p in plans),
         "active_peak_bytes": max(p["max_live_bytes"] for p in plans),
         "torch_allocated_peak_bytes": torch.cuda.max_memory_allocated() - base_alloc,
-        "torch_reserved_peak_bytes": torch.cuda.max_memory_reserved() - base_reserved,
+        "torch_reserved_peak_bytes": reserved_peak,
         "allocator": os.environ.get("PYTORCH_CUDA_ALLOC_CONF", "default (caching allocator)"),
     }
-    out["utilisation_torch"] = out["active_peak_bytes"] / out["torch_reserved_peak_bytes"]
+    out["utilisation_torch"] = out["active_peak_bytes"] / max(out["torch_reserved_peak_bytes"], 1)
     out["utilisation_static"] = out["active_peak_bytes"] / out["static_arena_bytes"]
     return out
 
