@@ -17,22 +17,23 @@
 //   * a score row is split between two threads (64 keys each): 16 softmax warps per SM, four per
 //     scheduler, each working through its 64 scores in chunks of 16 with the next chunk on its
 //     way from TMEM;
-//   * no running maximum.  A row's reference exponent is the largest score of its first key
-//     block; later probabilities are formed against it whatever their size -- fp32 sums and bf16
-//     probabilities keep their relative precision up to 2^90 -- so nothing is ever rescaled and
-//     the two threads of a row need not talk to each other inside the loop.  A row that does
-//     exceed 2^90 (scores far above everything its first 128 keys showed), or that hands the
-//     exponential polynomial an argument outside its range, is flagged, and its CTA runs two more
-//     sweeps: one that only takes the true row maximum, one that repeats the pass with that
-//     maximum as the reference of the flagged rows and with the polynomial's arguments clamped.
-//     Rows that were not flagged repeat exactly what they did before, bit for bit;
-//   * the scores leave the tensor core as finished exponents.  q arrives multiplied by
+//   * no running maximum and, in the normal pass, no reference at all.  q arrives multiplied by
 //     log2(e) / sqrt(64) (the Q projection's epilogue does that before its one rounding to bf16;
-//     a plain q is multiplied here, in shared memory), and from the second key block on the
-//     contraction has a fifth 16-wide step over [-reference, 0, ...] x [1, 0, ...] -- two small
-//     constant-shaped operands next to Q and K in shared memory, the reference (as a bf16
-//     number) written there by the row's thread -- so S = q k - reference and a softmax thread's
-//     work per pair of scores is the exponential, one packed add for the row sum and one pack.
+//     a plain q is multiplied here, in shared memory), so a score leaves the tensor core as the
+//     exponent to base 2 of its unnormalised probability and p = 2^s is formed whatever its size
+//     -- fp32 sums and bf16 probabilities keep their relative precision from 2^-90 to 2^90 -- so
+//     nothing is ever rescaled, the two threads of a row need not talk to each other inside the
+//     loop, and a softmax thread's work per pair of scores is the exponential, one packed add
+//     for the row sum and one pack.  A row that leaves that range (a probability of 2^90 or more,
+//     a row sum of 2^-90 or less), or that hands the exponential polynomial an argument outside
+//     its range, is flagged, and its CTA runs two more sweeps: one that only takes the true row
+//     maximum, one that repeats the pass with that maximum as the reference of the flagged rows
+//     and with the polynomial's arguments clamped.  In that repeat the reference is taken off
+//     inside the tensor core: the contraction gets a fifth 16-wide step over
+//     [-reference, 0, ...] x [1, 0, ...] -- two small constant-shaped operands next to Q and K in
+//     shared memory, the reference (as a bf16 number, zero for the rows that were fine) written
+//     there by the row's thread.  Rows that were not flagged repeat exactly what they did
+//     before, bit for bit;
 //
 //   warp 0      TMA producer: both Q tiles once, then K and V tiles through a ring of stages
 //   warp 1      owns TMEM; converged warp, one elected lane issues S(j+1) of a tile as soon as
@@ -73,6 +74,7 @@ constexpr int SMEM_BYTES = OFF_BAR + 512;
 constexpr int TMEM_COLS = 512;   // per tile 256: S [0,128), P [128,192), O [192,256)
 constexpr int TM_P = 128, TM_O = 192, TM_TILE = 256;
 constexpr float DANGER = 1.2379400392853803e27f;   // 2^90
+constexpr float TINY = 8.077935669463161e-28f;     // 2^-90
 // Share of the exponentials evaluated as a polynomial on the FMA pipe instead of the MUFU: three
 // column pairs of every eight (fixed positions).  Measured on B200 at 17776 x 17776 x 48 heads:
 // none 753, 1/8 808, 1/4 870, 3/8 929, 1/2 790 TFLOP/s (before later changes that added ~6 %).
@@ -96,22 +98,19 @@ __device__ __forceinline__ f32x2 exp2_poly_unclamped(f32x2 x2) {
                      __uint_as_float(__float_as_uint(p2.y) + (__float_as_uint(t2.y) << 23)));
 }
 
-// p = 2^(s + nm) for 16 consecutive score columns: 8 packed bf16x2 words, the values added
+// p = 2^s for 16 consecutive score columns: 8 packed bf16x2 words, the values added
 // into four packed partial sums.  POLY_NUM of every POLY_DEN column pairs (fixed positions)
 // evaluate 2^x as a polynomial on the FMA pipe, the others on the MUFU.  The polynomial is only
 // valid for arguments in [-125, 126].  SAFE = false: it is used as it is and `poly_abs` collects
 // the largest magnitude handed to it, for the caller to check afterwards.  SAFE = true:
 // arguments are clamped from below first (2^-125 stands in for zero); wherever the unclamped
 // form was valid the result has the same bits.
-template <bool SAFE, bool SHIFT>
-__device__ __forceinline__ void exp16(const float (&s)[16], f32x2 nm2, uint32_t (&pk)[8], f32x2 (&ls2)[4],
-                                      float& poly_abs) {
+template <bool SAFE>
+__device__ __forceinline__ void exp16(const float (&s)[16], uint32_t (&pk)[8], f32x2 (&ls2)[4], float& poly_abs) {
 #pragma unroll
   for (int t = 0; t < 16; t += 2) {
     const int pair = t >> 1;
-    // SHIFT: the scores still need the row's reference taken off (first key block); otherwise
-    // they come out of the tensor core as exponents already
-    f32x2 e2 = SHIFT ? add_f32x2(pack_f32x2(s[t], s[t + 1]), nm2) : pack_f32x2(s[t], s[t + 1]);
+    f32x2 e2 = pack_f32x2(s[t], s[t + 1]);   // the scores come out of the tensor core as exponents
     float e0, e1;
     if ((pair % POLY_DEN) < POLY_NUM) {
       if (SAFE) {
@@ -249,7 +248,7 @@ attention_dh64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
   const uint32_t o_tmem = t_lane + TM_O + half * (DH / 2);
   uint32_t sfull_ph = 0, pv_ph = 0, xch_ph = 0;
   int xch_slot = 0;
-  float m_ref = 0.f, neg_ref = 0.f, l_half = 0.f, m_true = -INFINITY;
+  float m_ref = 0.f, l_half = 0.f, m_true = -INFINITY;
   bool danger = false, danger_row = false;
   bool ok = true;
 
@@ -265,8 +264,8 @@ attention_dh64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
     return got ? base[(half ^ 1) * BM + r] : mine;
   };
 
-  // Sweep 0: the pass itself (reference = maximum of the first key block).  If a row overflowed:
-  // sweep 1 takes the true maximum of every row (scores only), sweep 2 repeats the pass.
+  // Sweep 0: the pass itself (no reference).  If a row left the safe range: sweep 1 takes the
+  // true maximum of every row (scores only), sweep 2 repeats the pass against it.
   for (int sweep = 0; sweep < 3; ++sweep) {
     const bool scores_only = (sweep == 1);
     if (warp == 0) {
@@ -313,8 +312,8 @@ attention_dh64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
       const uint64_t k_desc0 = smem_desc_sw128(smem_u32(smem + OFF_K), 16, 1024);
       const uint64_t qx_desc0 = smem_desc_sw128(smem_u32(smem + OFF_QX), 16, 1024);
       const uint64_t kx_desc = smem_desc_sw128(smem_u32(smem + OFF_KX), 16, 1024);
-      // with_ref: one more 16-wide step of the contraction, over [-reference, 0, ...] x [1, 0, ...]:
-      // the scores arrive with the row's reference already taken off
+      // with_ref (the repeat after a flag): one more 16-wide step of the contraction, over
+      // [-reference, 0, ...] x [1, 0, ...]: the scores arrive with the row's reference taken off
       auto issue_s = [&](int t, uint64_t k_desc, bool with_ref) {   // elected lane only
         const uint32_t d = tmem_base + t * TM_TILE;
         const uint64_t q_desc = q_desc0 + (uint64_t)(t * (Q_TILE_BYTES >> 4));
@@ -338,7 +337,7 @@ attention_dh64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
           }
           tc_fence_after();
           if (elect_one()) {
-            issue_s(t, k_desc, j > 0 && !scores_only);
+            issue_s(t, k_desc, sweep == 2);
             if (t == TILES - 1) mma_commit(&k_empty[k_st]);
           }
           __syncwarp();
@@ -383,8 +382,7 @@ attention_dh64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
         // one is used everywhere), negated, into column 0 of the extension operand
         const __nv_bfloat16 q = __float2bfloat16_rn(m_ref);
         m_ref = __bfloat162float(q);
-        neg_ref = -m_ref;
-        if (half == 0) *ref_slot = __float2bfloat16_rn(neg_ref);
+        if (half == 0) *ref_slot = __float2bfloat16_rn(-m_ref);
         fence_proxy_async_smem();
       };
       if (sweep == 0) {
@@ -444,18 +442,7 @@ attention_dh64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
           m_true = fmaxf(m_true, mine);
         }
       } else {
-        // (the new reference of a flagged row was published at the end of the second sweep)
-        if (sweep == 0) {
-          // the row's reference exponent: the largest score of its first key block
-          ok = mbar_wait_warp(&s_full[tile], sfull_ph, abort_flag);
-          if (ok) {
-            tc_fence_after();
-            const float mine = half_max(0);
-            m_ref = fmaxf(mine, exchange(mine));
-            publish_ref();
-          }
-        }
-        const f32x2 nm2 = pack_f32x2(neg_ref, neg_ref);
+        // (the reference of a flagged row was published at the end of the second sweep)
         // partial row sums and the largest polynomial argument of the whole sweep
         f32x2 ls2[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
         float poly_abs = 0.f;
@@ -466,14 +453,12 @@ attention_dh64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
         // previous block ended and has had this block's arithmetic to finish.
         auto run_block = [&](int j, auto masked_tag, auto first_tag, auto safe_tag) {
           constexpr bool MASKED = decltype(masked_tag)::value;
-          constexpr bool FIRST = decltype(first_tag)::value;
+          constexpr bool FIRST = decltype(first_tag)::value;   // no earlier product to wait for
           // the ragged last block masks with minus infinity, which the unclamped polynomial cannot take
           constexpr bool SAFE = decltype(safe_tag)::value || MASKED;
-          if (!(FIRST && sweep == 0)) {        // the first block of sweep 0 was waited for above
-            ok = mbar_wait_warp(&s_full[tile], sfull_ph, abort_flag);
-            if (!ok) return;
-            tc_fence_after();
-          }
+          ok = mbar_wait_warp(&s_full[tile], sfull_ph, abort_flag);
+          if (!ok) return;
+          tc_fence_after();
           sfull_ph ^= 1;
           const int valid = MASKED ? p.keys - j * BN - half * HALF : HALF;
           uint32_t pk[32];
@@ -486,17 +471,17 @@ attention_dh64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
           tmem_ld_wait_on(u16(b1));
           tmem_ld_wait_on(u16(b2));
           if (MASKED && valid < 16) mask_tail16(b0, valid);
-          exp16<SAFE, FIRST>(b0, nm2, pk8(0), ls2, poly_abs);
+          exp16<SAFE>(b0, pk8(0), ls2, poly_abs);
           tmem_ld16(s_tmem + 48, u16(b0));
           if (MASKED && valid < 32) mask_tail16(b1, valid - 16);
-          exp16<SAFE, FIRST>(b1, nm2, pk8(1), ls2, poly_abs);
+          exp16<SAFE>(b1, pk8(1), ls2, poly_abs);
           tmem_ld_wait_on(u16(b0));
           tc_fence_before();
           mbar_arrive(&s_free[tile]);                       // S(j) is in registers: S(j+1) may land
           if (MASKED && valid < 48) mask_tail16(b2, valid - 32);
-          exp16<SAFE, FIRST>(b2, nm2, pk8(2), ls2, poly_abs);
+          exp16<SAFE>(b2, pk8(2), ls2, poly_abs);
           if (MASKED) mask_tail16(b0, valid - 48);
-          exp16<SAFE, FIRST>(b0, nm2, pk8(3), ls2, poly_abs);
+          exp16<SAFE>(b0, pk8(3), ls2, poly_abs);
           if (!FIRST) {
             if (!mbar_peek(&pv_done[tile], pv_ph)) ok = mbar_wait_warp(&pv_done[tile], pv_ph, abort_flag);
             pv_ph ^= 1;
@@ -533,7 +518,12 @@ attention_dh64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
         danger = !(l_half < DANGER) || poly_abs > 120.f;
       }
       if (ok && sweep == 0) {
-        danger_row = (exchange(danger ? 1.f : 0.f) != 0.f) || danger;
+        // The row's sum (an infinity stands for a thread's own flag): above 2^90 a probability
+        // overflowed or came close; at or below 2^-90 the row's scores lie so far below zero that
+        // the small terms were flushed away.  Both threads of the row come to the same verdict.
+        const float mine = danger ? INFINITY : l_half;
+        const float l_row = mine + exchange(mine);
+        danger_row = !(l_row < DANGER) || !(l_row > TINY);
         if (danger_row) *danger_any = 1;
       }
       if (ok && sweep == 1) {

@@ -298,6 +298,45 @@ def test_gemm_epilogue_rmsnorm_rope(name, norm_all):
     assert_bf16_close(from_dev_bf16(out), ref, ("gemm norm+rope", name, norm_all), atol_rms=3e-4)
 
 
+@pytest.mark.parametrize("offset", [-260.0, -100.0, 100.0, 260.0])
+def test_attention_dh64_scores_far_from_zero(offset):
+    """Every score of a row lies near `offset` (in exponents to base 2), with a spread of a few
+    units: far below zero the unnormalised probabilities underflow, far above they overflow, and
+    in between (|offset| = 100) the sums leave the range the kernel trusts.  The head_dim-64
+    kernel forms 2^score without a reference in its first pass, so all of these must be caught
+    by its range check and repeated against the row's true maximum; rows of an ordinary head in
+    the same launch are unaffected."""
+    rng = np.random.default_rng(91)
+    B, rows, keys, H, dh = 1, 300, 700, 2, 64
+    D = H * dh
+    u = rng.standard_normal(dh)
+    u /= np.linalg.norm(u)
+    q = rng.standard_normal((B, rows, D))
+    kv = rng.standard_normal((B, keys, 2 * D))
+    # head 0: q = a u + noise, k = b u + noise with a * b / 8 * log2(e) = offset
+    a = 30.0
+    b = offset * 8.0 / 1.4426950408889634 / a
+    q[0, :, :dh] = a * u + 0.3 * rng.standard_normal((rows, dh))
+    kv[0, :, :dh] = b * u + 0.3 * rng.standard_normal((keys, dh))
+    (qb, qf), kvb = _exponent_units(q, dh), bf16_bits(kv.astype(np.float32))
+    kvf = bits_to_f64(kvb)
+    q_dev, kv_dev = to_dev(qb), to_dev(kvb)
+    o = torch.zeros(B, rows, D, dtype=torch.int16, device=DEV)
+    lse = torch.zeros(B, H, rows, dtype=torch.float32, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    xb.xema_op_attention(q_dev.data_ptr(), D, rows, kv_dev.data_ptr(), kv_dev.data_ptr() + D * 2, 2 * D, keys,
+                         o.data_ptr(), lse.data_ptr(), B, rows, keys, H, dh, status=status.data_ptr(), q_scale=1.0)
+    _sync_status(status)
+    got = from_dev_bf16(o)
+    expo = (qf[0, :, :dh] @ kvf[0, :, :dh].T) / math.sqrt(dh) * 1.4426950408889634
+    assert abs(np.median(expo) - offset) < 0.1 * abs(offset) and expo.max() - expo.min() > 10
+    for h in range(H):
+        ref_o, ref_l = ob.attention_head(qf[0, :, h * dh:(h + 1) * dh], kvf[0, :, h * dh:(h + 1) * dh],
+                                         kvf[0, :, D + h * dh:D + (h + 1) * dh], 1 / math.sqrt(dh))
+        assert_bf16_close(got[0, :, h * dh:(h + 1) * dh], ref_o, ("scores far from zero", offset, h), atol_rms=2e-2, cos=0.9999)
+        assert np.abs(lse.cpu().numpy()[0, h] - ref_l).max() < 1e-3 * max(np.abs(ref_l).max(), 1.0)
+
+
 @pytest.mark.parametrize("dh", [64, 128])
 def test_attention_scores_growing_along_the_keys(dh):
     """Keys whose scores rise steadily with the key index: the running max moves by more than
