@@ -101,11 +101,12 @@ __device__ __forceinline__ f32x2 exp2_poly_unclamped(f32x2 x2) {
 // p = 2^s for 16 consecutive score columns: 8 packed bf16x2 words, the values added
 // into four packed partial sums.  POLY_NUM of every POLY_DEN column pairs (fixed positions)
 // evaluate 2^x as a polynomial on the FMA pipe, the others on the MUFU.  The polynomial is only
-// valid for arguments in [-125, 126].  SAFE = false: it is used as it is and `poly_abs` collects
-// the largest magnitude handed to it, for the caller to check afterwards.  SAFE = true:
+// valid for arguments in [-125, 126].  SAFE = false: it is used as it is and, with TRACK,
+// `poly_abs` collects the largest magnitude handed to it, for the caller to check afterwards
+// (without TRACK the caller knows a bound on every score beforehand).  SAFE = true:
 // arguments are clamped from below first (2^-125 stands in for zero); wherever the unclamped
 // form was valid the result has the same bits.
-template <bool SAFE>
+template <bool SAFE, bool TRACK>
 __device__ __forceinline__ void exp16(const float (&s)[16], uint32_t (&pk)[8], f32x2 (&ls2)[4], float& poly_abs) {
 #pragma unroll
   for (int t = 0; t < 16; t += 2) {
@@ -116,7 +117,7 @@ __device__ __forceinline__ void exp16(const float (&s)[16], uint32_t (&pk)[8], f
       if (SAFE) {
         e2 = exp2_poly_f32x2(e2);
       } else {
-        poly_abs = max3(poly_abs, fabsf(e2.x), fabsf(e2.y));
+        if (TRACK) poly_abs = max3(poly_abs, fabsf(e2.x), fabsf(e2.y));
         e2 = exp2_poly_unclamped(e2);
       }
       unpack_f32x2(e2, e0, e1);
@@ -164,6 +165,7 @@ struct Attn64Params {
   int batch, rows, keys, heads;
   float q_scale;      // q k^T times this = exponents to base 2 (1: q arrives already multiplied)
   unsigned int* status;
+  const __nv_bfloat16 *gain_q, *gain_k;   // RMSNorm gains behind q and k, or null (see AttnLaunch)
 };
 
 __global__ void __launch_bounds__(THREADS, 1)
@@ -185,6 +187,7 @@ attention_dh64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 34);
   volatile uint32_t* abort_flag = tmem_slot + 1;
   volatile uint32_t* danger_any = tmem_slot + 2;
+  uint32_t* gain_max = tmem_slot + 3;          // [2] bit patterns of max|gain_q|, max|gain_k|
   volatile float* xch = reinterpret_cast<volatile float*>(smem + OFF_XCH);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -214,6 +217,7 @@ attention_dh64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
     mbar_init(q_ready, 32 * SOFTMAX_WARPS);
     *abort_flag = 0;
     *danger_any = 0;
+    gain_max[0] = gain_max[1] = 0;
     fence_mbar_init();
     prefetch_tmap(&map_q);
     prefetch_tmap(&map_k);
@@ -250,6 +254,7 @@ attention_dh64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
   int xch_slot = 0;
   float m_ref = 0.f, l_half = 0.f, m_true = -INFINITY;
   bool danger = false, danger_row = false;
+  bool bounded = false;      // every score is known to lie well inside the polynomial's range
   bool ok = true;
 
   // One value from each of the two threads that share a row; returns the partner's.
@@ -415,6 +420,20 @@ attention_dh64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
           fence_proxy_async_smem();
           mbar_arrive(q_ready);
         }
+        // With q and k out of an RMSNorm (gains g), a rotation and, for q, the factor log2(e) / 8,
+        // a head of q has norm <= max|g_q| * log2(e) and a head of k norm <= 8 * max|g_k|: every
+        // score lies within +-11.55 * max|g_q| * max|g_k| (plus the bf16 roundings, under half a
+        // percent).  Far inside the polynomial's range nothing needs to be tracked per score.
+        if (p.gain_q && p.gain_k && p.q_scale == 1.f) {
+          if (ts < DH) {
+            atomicMax(&gain_max[0], __float_as_uint(fabsf(__bfloat162float(p.gain_q[ts]))));
+            atomicMax(&gain_max[1], __float_as_uint(fabsf(__bfloat162float(p.gain_k[ts]))));
+          }
+          asm volatile("bar.sync 1, %0;" ::"n"(32 * SOFTMAX_WARPS) : "memory");
+          const float gq = __uint_as_float(*(volatile uint32_t*)&gain_max[0]);
+          const float gk = __uint_as_float(*(volatile uint32_t*)&gain_max[1]);
+          bounded = gq * gk * 11.55f * 1.01f < 100.f;    // false for a NaN gain
+        }
       }
       auto u16 = [](float(&a)[16]) -> uint32_t(&)[16] { return *reinterpret_cast<uint32_t(*)[16]>(&a[0]); };
       auto u32 = [](float(&a)[32]) -> uint32_t(&)[32] { return *reinterpret_cast<uint32_t(*)[32]>(&a[0]); };
@@ -451,7 +470,8 @@ attention_dh64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
         // S(j+1) may land -- when half of the block is done.  P(j) goes to TMEM in one piece at
         // the end: O += P(j-1) V(j-1), which reads the same columns, was only issued when the
         // previous block ended and has had this block's arithmetic to finish.
-        auto run_block = [&](int j, auto masked_tag, auto first_tag, auto safe_tag) {
+        auto run_block = [&](int j, auto masked_tag, auto first_tag, auto safe_tag, auto track_tag) {
+          constexpr bool TRACK = decltype(track_tag)::value;
           constexpr bool MASKED = decltype(masked_tag)::value;
           constexpr bool FIRST = decltype(first_tag)::value;   // no earlier product to wait for
           // the ragged last block masks with minus infinity, which the unclamped polynomial cannot take
@@ -471,17 +491,17 @@ attention_dh64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
           tmem_ld_wait_on(u16(b1));
           tmem_ld_wait_on(u16(b2));
           if (MASKED && valid < 16) mask_tail16(b0, valid);
-          exp16<SAFE>(b0, pk8(0), ls2, poly_abs);
+          exp16<SAFE, TRACK>(b0, pk8(0), ls2, poly_abs);
           tmem_ld16(s_tmem + 48, u16(b0));
           if (MASKED && valid < 32) mask_tail16(b1, valid - 16);
-          exp16<SAFE>(b1, pk8(1), ls2, poly_abs);
+          exp16<SAFE, TRACK>(b1, pk8(1), ls2, poly_abs);
           tmem_ld_wait_on(u16(b0));
           tc_fence_before();
           mbar_arrive(&s_free[tile]);                       // S(j) is in registers: S(j+1) may land
           if (MASKED && valid < 48) mask_tail16(b2, valid - 32);
-          exp16<SAFE>(b2, pk8(2), ls2, poly_abs);
+          exp16<SAFE, TRACK>(b2, pk8(2), ls2, poly_abs);
           if (MASKED) mask_tail16(b0, valid - 48);
-          exp16<SAFE>(b0, pk8(3), ls2, poly_abs);
+          exp16<SAFE, TRACK>(b0, pk8(3), ls2, poly_abs);
           if (!FIRST) {
             if (!mbar_peek(&pv_done[tile], pv_ph)) ok = mbar_wait_warp(&pv_done[tile], pv_ph, abort_flag);
             pv_ph ^= 1;
@@ -494,18 +514,19 @@ attention_dh64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
           mbar_arrive(&p_full[tile]);
         };
         const int n_full = p.keys / BN;                     // blocks without keys past the end
-        auto run_all = [&](auto safe_tag) {
+        auto run_all = [&](auto safe_tag, auto track_tag) {
           if (ok) {
-            if (n_full > 0) run_block(0, std::false_type{}, std::true_type{}, safe_tag);
-            else run_block(0, std::true_type{}, std::true_type{}, safe_tag);
+            if (n_full > 0) run_block(0, std::false_type{}, std::true_type{}, safe_tag, track_tag);
+            else run_block(0, std::true_type{}, std::true_type{}, safe_tag, track_tag);
           }
-          for (int j = 1; ok && j < n_full; ++j) run_block(j, std::false_type{}, std::false_type{}, safe_tag);
-          if (ok && n_full > 0 && n_full < n_kv) run_block(n_full, std::true_type{}, std::false_type{}, safe_tag);
+          for (int j = 1; ok && j < n_full; ++j) run_block(j, std::false_type{}, std::false_type{}, safe_tag, track_tag);
+          if (ok && n_full > 0 && n_full < n_kv) run_block(n_full, std::true_type{}, std::false_type{}, safe_tag, track_tag);
         };
         // the repeat after an overflow clamps the polynomial's arguments (rows that were fine get
         // the same bits from either form)
-        if (sweep == 0) run_all(std::false_type{});
-        else run_all(std::true_type{});
+        if (sweep != 0) run_all(std::true_type{}, std::false_type{});
+        else if (bounded) run_all(std::false_type{}, std::false_type{});
+        else run_all(std::false_type{}, std::true_type{});
         // the accumulator is final once the last products have finished
         if (ok) {
           ok = mbar_wait_warp(&pv_done[tile], pv_ph, abort_flag);
@@ -585,6 +606,8 @@ int launch_attention_dh64(const AttnLaunch& a, cudaStream_t stream) {
   p.heads = a.heads;
   p.q_scale = a.q_scale;
   p.status = a.status;
+  p.gain_q = (const __nv_bfloat16*)a.gain_q;
+  p.gain_k = (const __nv_bfloat16*)a.gain_k;
   dim3 grid((a.rows + TILES * BM - 1) / (TILES * BM), a.heads, a.batch);
   attention_dh64_kernel<<<grid, THREADS, SMEM_BYTES, stream>>>(a.map_q, a.map_k, a.map_v, p);
   return check_launch();

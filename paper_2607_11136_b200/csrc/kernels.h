@@ -95,6 +95,13 @@ struct AttnLaunch {
   // q, 1 if q was already multiplied by that (as the fused epilogue of the Q projection does)
   float q_scale;
   unsigned int* status;
+  // head_dim 64 only, both or neither: the RMSNorm gains (bf16 [head_dim], device) that q and k
+  // went through before their rotation, with q multiplied by log2(e) / sqrt(head_dim) afterwards
+  // (q_scale = 1).  A head of q then has norm <= max|gain_q| * log2(e) and a head of k norm <=
+  // max|gain_k| * sqrt(head_dim), which bounds every score; where that bound is small the kernel
+  // skips its per-score range tracking.  Null: nothing is known about the scores.
+  const void* gain_q;
+  const void* gain_k;
 };
 int attn_prepare(AttnLaunch* a, const void* q, long long ldq, long long q_batch_rows, const void* k, const void* v,
                  long long ldkv, long long kv_batch_rows);

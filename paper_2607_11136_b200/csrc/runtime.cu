@@ -519,6 +519,7 @@ int xema_plan_bind(xema_plan* plan, void* arena_dev, uint64_t arena_bytes, const
       tag(a, "ATTN", ci, 4.0 * Bd * n * Sd * Dd, 4.0 * Bd * n * Dd + 4.0 * Bd * Sd * Dd + 4.0 * Bd * c.heads * n);
       a.attn.o = o_t; a.attn.lse = lse; a.attn.batch = pc.nb; a.attn.rows = n; a.attn.keys = (int)S_all;
       a.attn.heads = c.heads; a.attn.head_dim = c.head_dim; a.attn.status = status; a.attn.q_scale = 1.f;
+      a.attn.gain_q = w.g_q; a.attn.gain_k = w.g_k;     // q and k come out of the fused RMSNorm + RoPE epilogues
       rc = attn_prepare(&a.attn, q, D, n, kv_b, kv_b + D * 2, 2 * D, S_all);
       if (rc) return rc;
       plan->ops.push_back(a);
