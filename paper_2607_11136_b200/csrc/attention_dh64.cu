@@ -541,7 +541,7 @@ attention_dh64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
       if (ok && sweep == 0) {
         // The row's sum (an infinity stands for a thread's own flag): above 2^90 a probability
         // overflowed or came close; at or below 2^-90 the row's scores lie so far below zero that
-        // the small terms were flushed away.  Both threads of the row come to the same verdict.
+        // the small terms were flushed away.  Both threads of the row decide the same.
         const float mine = danger ? INFINITY : l_half;
         const float l_row = mine + exchange(mine);
         danger_row = !(l_row < DANGER) || !(l_row > TINY);
