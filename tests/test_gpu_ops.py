@@ -337,6 +337,36 @@ def test_attention_dh64_scores_far_from_zero(offset):
         assert np.abs(lse.cpu().numpy()[0, h] - ref_l).max() < 1e-3 * max(np.abs(ref_l).max(), 1.0)
 
 
+def test_attention_dh64_rows_keep_their_bits_when_neighbours_repeat():
+    """Rows 128..255 of a CTA get scores in the hundreds and make the whole CTA repeat its pass;
+    rows 0..127 of the same CTA (and the rows of the next CTA) must come out with exactly the
+    bits they have when nothing repeats."""
+    rng = np.random.default_rng(17)
+    B, rows, keys, H, dh = 1, 384, 900, 1, 64
+    q = rng.standard_normal((B, rows, dh))
+    kv = rng.standard_normal((B, keys, 2 * dh))
+    loud = q.copy()
+    loud[0, 128:256] *= 60.0                                   # exponents of +-300 and more
+    kvb = bf16_bits(kv.astype(np.float32))
+    kv_dev = to_dev(kvb)
+    outs = []
+    for qq in (q, loud):
+        qb, _ = _exponent_units(qq, dh)
+        q_dev = to_dev(qb)
+        o = torch.zeros(B, rows, dh, dtype=torch.int16, device=DEV)
+        lse = torch.zeros(B, H, rows, dtype=torch.float32, device=DEV)
+        status = torch.zeros(1, dtype=torch.int32, device=DEV)
+        xb.xema_op_attention(q_dev.data_ptr(), dh, rows, kv_dev.data_ptr(), kv_dev.data_ptr() + dh * 2, 2 * dh, keys,
+                             o.data_ptr(), lse.data_ptr(), B, rows, keys, H, dh, status=status.data_ptr(), q_scale=1.0)
+        _sync_status(status)
+        outs.append((o.cpu().numpy(), lse.cpu().numpy()))
+    (o0, l0), (o1, l1) = outs
+    quiet = np.r_[0:128, 256:rows]
+    assert np.array_equal(o0[:, quiet], o1[:, quiet]) and np.array_equal(l0[:, :, quiet], l1[:, :, quiet])
+    assert not np.array_equal(o0[:, 128:256], o1[:, 128:256])
+    assert np.isfinite(l1).all()
+
+
 @pytest.mark.parametrize("dh", [64, 128])
 def test_attention_scores_growing_along_the_keys(dh):
     """Keys whose scores rise steadily with the key index: the running max moves by more than
